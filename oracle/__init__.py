@@ -1,0 +1,6 @@
+"""fp64 CPU oracle for the gated delta-rule prefill — test infrastructure only.
+
+Nothing in the product package may import this; only the tests, the smoke check
+and the CPU-baseline leg of the benchmark do.
+"""
+from .gdn_oracle import (chunked, dense, num_threads, sequential)  # noqa: F401

@@ -1,0 +1,29 @@
+"""Build the fp64 CPU oracle (test infrastructure) into oracle/libgdn_oracle.so.
+
+Plain g++ with OpenMP; no CUDA, no torch.  Run as ``python oracle/build.py`` or
+call ``build()``; the shared object is rebuilt only when the source is newer.
+"""
+from __future__ import annotations
+
+import os
+import subprocess
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+SRC = os.path.join(HERE, "gdn_oracle.cpp")
+LIB = os.path.join(HERE, "libgdn_oracle.so")
+
+
+def build(force: bool = False) -> str:
+    if (not force and os.path.exists(LIB)
+            and os.path.getmtime(LIB) >= os.path.getmtime(SRC)):
+        return LIB
+    tmp = LIB + f".tmp{os.getpid()}"
+    cmd = ["g++", "-O2", "-std=c++17", "-fopenmp", "-fPIC", "-shared",
+           "-ffp-contract=off", "-o", tmp, SRC]
+    subprocess.run(cmd, check=True)
+    os.replace(tmp, LIB)
+    return LIB
+
+
+if __name__ == "__main__":
+    print(build(force=True))

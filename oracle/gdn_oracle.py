@@ -1,0 +1,106 @@
+"""ctypes front end of the fp64 CPU oracle (test infrastructure only).
+
+Every function takes numpy arrays of any float dtype, widens them exactly to
+fp64, and returns ``(out, final_state)`` as fp64 arrays.  Layouts are those of
+the C file: ``q,k [B,T,H,d_k]``, ``v [B,T,H,d_v]``, ``log_alpha,beta [B,T,H]``,
+``initial_state [N,H,d_k,d_v]``; with ``cu_seqlens`` the tensors are packed
+``[T_total,H,.]`` and ``N = len(cu_seqlens) - 1``.
+
+  sequential  the token-by-token recurrence (the definition; Section "A chunked
+              delta-rule scan for the recurrent layers")
+  chunked     the intra-/inter-chunk form of the same section (form=1: its
+              S' = M S + N variant)
+  dense       the whole sequence as one general linear system (brute force)
+"""
+from __future__ import annotations
+
+import ctypes
+
+import numpy as np
+
+from . import build as _build
+
+_lib = None
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        lib = ctypes.CDLL(_build.build())
+        dp = ctypes.POINTER(ctypes.c_double)
+        ip = ctypes.POINTER(ctypes.c_int32)
+        common = [dp, dp, dp, dp, dp, dp, dp, dp, ip] + [ctypes.c_int] * 5
+        lib.gdn_oracle_sequential.argtypes = common
+        lib.gdn_oracle_dense.argtypes = common
+        lib.gdn_oracle_chunked.argtypes = common + [ctypes.c_int, ctypes.c_int]
+        for f in (lib.gdn_oracle_sequential, lib.gdn_oracle_dense, lib.gdn_oracle_chunked,
+                  lib.gdn_oracle_num_threads):
+            f.restype = ctypes.c_int
+        _lib = lib
+    return _lib
+
+
+def num_threads() -> int:
+    return int(_load().gdn_oracle_num_threads())
+
+
+def _f64(x):
+    return np.ascontiguousarray(np.asarray(x), dtype=np.float64)
+
+
+def _ptr(x):
+    return None if x is None else x.ctypes.data_as(ctypes.POINTER(ctypes.c_double))
+
+
+def _prepare(q, k, v, log_alpha, beta, initial_state, cu_seqlens):
+    q, k, v, a, b = (_f64(x) for x in (q, k, v, log_alpha, beta))
+    if cu_seqlens is None:
+        if q.ndim != 4:
+            raise ValueError("q must be [B,T,H,d_k] without cu_seqlens")
+        B, T, H, dk = q.shape
+        N = B
+        cu = None
+    else:
+        if q.ndim != 3:
+            raise ValueError("q must be packed [T,H,d_k] with cu_seqlens")
+        T, H, dk = q.shape
+        cu = np.ascontiguousarray(np.asarray(cu_seqlens), dtype=np.int32)
+        B = N = cu.shape[0] - 1
+    dv = v.shape[-1]
+    if k.shape != q.shape or v.shape[:-1] != q.shape[:-1]:
+        raise ValueError("q, k, v shapes disagree")
+    if a.shape != q.shape[:-1] or b.shape != q.shape[:-1]:
+        raise ValueError("gate shapes disagree with q")
+    s0 = None
+    if initial_state is not None:
+        s0 = _f64(initial_state)
+        if s0.shape != (N, H, dk, dv):
+            raise ValueError("initial_state must be [N,H,d_k,d_v]")
+    out = np.empty(v.shape, dtype=np.float64)
+    fin = np.empty((N, H, dk, dv), dtype=np.float64)
+    return (q, k, v, a, b, s0, out, fin, cu), (B, T, H, dk, dv)
+
+
+def _call(fn, arrs, dims, *extra):
+    q, k, v, a, b, s0, out, fin, cu = arrs
+    cup = None if cu is None else cu.ctypes.data_as(ctypes.POINTER(ctypes.c_int32))
+    rc = fn(_ptr(q), _ptr(k), _ptr(v), _ptr(a), _ptr(b), _ptr(s0), _ptr(out), _ptr(fin),
+            cup, *dims, *extra)
+    if rc != 0:
+        raise ValueError(f"oracle rejected its arguments (code {rc})")
+    return out, fin
+
+
+def sequential(q, k, v, log_alpha, beta, initial_state=None, cu_seqlens=None):
+    arrs, dims = _prepare(q, k, v, log_alpha, beta, initial_state, cu_seqlens)
+    return _call(_load().gdn_oracle_sequential, arrs, dims)
+
+
+def chunked(q, k, v, log_alpha, beta, initial_state=None, cu_seqlens=None, chunk=64, form=0):
+    arrs, dims = _prepare(q, k, v, log_alpha, beta, initial_state, cu_seqlens)
+    return _call(_load().gdn_oracle_chunked, arrs, dims, int(chunk), int(form))
+
+
+def dense(q, k, v, log_alpha, beta, initial_state=None, cu_seqlens=None):
+    arrs, dims = _prepare(q, k, v, log_alpha, beta, initial_state, cu_seqlens)
+    return _call(_load().gdn_oracle_dense, arrs, dims)
