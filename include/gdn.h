@@ -1,0 +1,136 @@
+/*
+ * gdn.h -- C ABI of the B200 (sm_100a) chunked gated delta-rule prefill library.
+ *
+ * The operation.  For every sequence n and head h (all independent), with a
+ * recurrent state S in R^{d_k x d_v} per head (Section "The model": state
+ * S in R^{H_k x H_v} per value head, updated token by token) the library
+ * evaluates the gated delta-net recurrence of Section "A chunked delta-rule scan
+ * for the recurrent layers", S_t = diag(gamma_t) S_{t-1} + k_t delta_t^T, read as
+ *
+ *     S      <- exp(log_alpha_t) * S                 (scalar gate per token, head)
+ *     delta  <- beta_t * (v_t - S^T k_t)             (against the decayed state)
+ *     S      <- S + k_t delta^T
+ *     out_t  <- S^T q_t                              (updated state, no 1/sqrt(d_k))
+ *
+ * over a whole prompt, using the intra-/inter-chunk form of that section: per
+ * 64-token chunk a cumulative log gate, the decay-masked token-token matrices,
+ * a forward substitution of the unit lower triangular system, the WY factors,
+ * and a short recurrence over chunks that carries the state.  The result does
+ * not depend on the chunk size; `chunk` names the internal tiling and only 64
+ * is supported.
+ *
+ * Layouts (row-major, last index fastest; every pointer is a DEVICE pointer
+ * unless its name ends in _host, and must be 16-byte aligned):
+ *     q, k                       [B, T, H, d_k]
+ *     v, out                     [B, T, H, d_v]
+ *     log_alpha, beta            [B, T, H]            fp32
+ *     initial_state, final_state [B, H, d_k, d_v]     fp32
+ * With cu_seqlens != NULL the tensors are packed [T, H, .] where T is the total
+ * number of tokens, B is the number of sequences and sequence n owns tokens
+ * [cu_seqlens[n], cu_seqlens[n+1]); cu_seqlens has B+1 int32 entries,
+ * cu_seqlens[0] = 0, cu_seqlens[B] = T.  A sequence of length 0 passes its
+ * state through.  initial_state == NULL means zeros; final_state == NULL means
+ * "do not return it".  final_state may alias initial_state; no other input may
+ * alias an output.
+ *
+ * Ownership and execution.  The caller owns every buffer.  The calls enqueue
+ * work on `stream` and return without synchronising; they allocate no device
+ * memory.  All functions return a gdn_status (0 = success) and never abort.
+ * Nothing is launched when a non-zero status is returned for an argument error.
+ */
+#ifndef GDN_H_
+#define GDN_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    GDN_OK = 0,
+    GDN_ERR_INVALID_ARG = 1,  /* NULL required pointer, non-positive size, bad cu_seqlens_host */
+    GDN_ERR_UNSUPPORTED = 2,  /* chunk != 64, unsupported (d_k, d_v), misaligned pointer */
+    GDN_ERR_WORKSPACE = 3,    /* caller-provided scratch too small */
+    GDN_ERR_CUDA = 4,         /* a CUDA runtime/driver call or a launch failed */
+    GDN_ERR_TIMEOUT = 5       /* a bounded device-side wait expired (see gdn_query_status) */
+} gdn_status;
+
+/* Same handle as cudaStream_t / CUstream (NULL = the default stream). */
+typedef struct CUstream_st* gdn_stream_t;
+
+/*
+ * The chunked prefill, bf16 q/k/v/out, fp32 gates and state (the main entry
+ * point; steps: cumulative gate, decay-masked KK^T and QK^T, forward
+ * substitution, WY factors, inter-chunk state recurrence, output -- Section "A
+ * chunked delta-rule scan for the recurrent layers").  Supported: chunk = 64,
+ * d_k = 128, d_v a multiple of 128 (tensor-core path); other d_k, d_v that are
+ * multiples of 32 with d_k <= 128 fall back to the fp32-arithmetic kernel below.
+ */
+int gdn_chunk_prefill(const void* q, const void* k, const void* v,
+                      const float* log_alpha, const float* beta,
+                      const float* initial_state,
+                      void* out, float* final_state,
+                      const int32_t* cu_seqlens,
+                      int B, int T, int H, int d_k, int d_v, int chunk,
+                      gdn_stream_t stream);
+
+/*
+ * Same operation and argument list with fp32 q/k/v/out and fp32 arithmetic
+ * throughout (plain FMA kernels; the paper's own precision, Section "A chunked
+ * delta-rule scan for the recurrent layers").  Supported: chunk = 64, d_k and d_v
+ * multiples of 32, d_k <= 128.
+ */
+int gdn_chunk_prefill_f32(const float* q, const float* k, const float* v,
+                          const float* log_alpha, const float* beta,
+                          const float* initial_state,
+                          float* out, float* final_state,
+                          const int32_t* cu_seqlens,
+                          int B, int T, int H, int d_k, int d_v, int chunk,
+                          gdn_stream_t stream);
+
+/*
+ * bf16 q/k/v/out through the fp32-arithmetic kernel (inputs widened exactly, fp32
+ * everywhere inside, one rounding at the output).  A slow cross-check of the
+ * tensor-core path with the same chunked algorithm; same support as the f32 call.
+ */
+int gdn_chunk_prefill_bf16_simt(const void* q, const void* k, const void* v,
+                                const float* log_alpha, const float* beta,
+                                const float* initial_state,
+                                void* out, float* final_state,
+                                const int32_t* cu_seqlens,
+                                int B, int T, int H, int d_k, int d_v, int chunk,
+                                gdn_stream_t stream);
+
+/*
+ * The bf16 prefill with HOST buffers: copies the inputs to the device staging
+ * area (cudaMemcpyAsync on `stream`; pinned host memory keeps it asynchronous),
+ * runs gdn_chunk_prefill there and copies out/final_state back, all on `stream`,
+ * without synchronising.  staging_dev is caller-owned device memory of at least
+ * gdn_host_staging_bytes(...) bytes, 256-byte aligned.  cu_seqlens_host may be
+ * NULL; initial_state_host / final_state_host may be NULL as above.
+ * Errors: as gdn_chunk_prefill, plus GDN_ERR_WORKSPACE when staging is too small.
+ */
+int gdn_chunk_prefill_host(const void* q_host, const void* k_host, const void* v_host,
+                           const float* log_alpha_host, const float* beta_host,
+                           const float* initial_state_host,
+                           void* out_host, float* final_state_host,
+                           const int32_t* cu_seqlens_host,
+                           int B, int T, int H, int d_k, int d_v, int chunk,
+                           void* staging_dev, size_t staging_bytes,
+                           gdn_stream_t stream);
+
+/* Bytes of device staging gdn_chunk_prefill_host needs for these sizes (0 on bad sizes). */
+size_t gdn_host_staging_bytes(int B, int T, int H, int d_k, int d_v);
+
+/* Number of kernels this library has launched in this process so far. */
+unsigned long long gdn_launch_count(void);
+
+/* Static description of a status code. */
+const char* gdn_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GDN_H_ */

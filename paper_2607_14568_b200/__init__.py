@@ -1,0 +1,10 @@
+"""B200-native chunked gated delta-rule prefill: Python binding of the C-ABI library.
+
+The functions here only marshal arguments (pointers, sizes, the stream) into
+``libgdn.so``; every step of the computation runs in the library's CUDA kernels.
+There is no CPU fallback: importing works without the shared object (so that the
+build step can run), but any call raises if it is missing.
+"""
+from .binding import (GdnError, gdn_chunk_prefill, gdn_chunk_prefill_bf16_simt,  # noqa: F401
+                      gdn_chunk_prefill_f32, gdn_chunk_prefill_host, gdn_host_staging_bytes,
+                      gdn_launch_count, gdn_status_string, lib, lib_path)

@@ -1,0 +1,160 @@
+"""ctypes binding of libgdn.so.  Names and argument order follow include/gdn.h.
+
+Tensors are ``torch`` tensors (used only for device memory and streams); they are
+passed as raw pointers.  ``T`` is taken from the tensors: ``q`` is ``[B,T,H,d_k]``,
+or packed ``[T,H,d_k]`` when ``cu_seqlens`` (an int32 tensor with one entry more
+than there are sequences) is given.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "libgdn.so")
+_lib = None
+
+
+class GdnError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: status {status} ({gdn_status_string(status)})")
+
+
+def lib_path() -> str:
+    return _LIB_PATH
+
+
+def lib():
+    """The loaded library; raises if it has not been built (no fallback)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(_LIB_PATH):
+            raise RuntimeError(f"{_LIB_PATH} is missing: build it with "
+                               "`python -m paper_2607_14568_b200.build` (there is no CPU fallback)")
+        L = ctypes.CDLL(_LIB_PATH)
+        vp, ip, i, sz = ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t
+        prefill = [vp] * 8 + [ip] + [i] * 6 + [vp]
+        for name in ("gdn_chunk_prefill", "gdn_chunk_prefill_f32", "gdn_chunk_prefill_bf16_simt"):
+            getattr(L, name).argtypes = prefill
+            getattr(L, name).restype = i
+        L.gdn_chunk_prefill_host.argtypes = [vp] * 8 + [ip] + [i] * 6 + [vp, sz, vp]
+        L.gdn_chunk_prefill_host.restype = i
+        L.gdn_host_staging_bytes.argtypes = [i] * 5
+        L.gdn_host_staging_bytes.restype = sz
+        L.gdn_launch_count.argtypes = []
+        L.gdn_launch_count.restype = ctypes.c_ulonglong
+        L.gdn_status_string.argtypes = [i]
+        L.gdn_status_string.restype = ctypes.c_char_p
+        _lib = L
+    return _lib
+
+
+def gdn_status_string(status: int) -> str:
+    return lib().gdn_status_string(int(status)).decode()
+
+
+def gdn_launch_count() -> int:
+    return int(lib().gdn_launch_count())
+
+
+def gdn_host_staging_bytes(B: int, T: int, H: int, d_k: int, d_v: int) -> int:
+    return int(lib().gdn_host_staging_bytes(B, T, H, d_k, d_v))
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _dims(q, v, cu_seqlens):
+    if cu_seqlens is None:
+        B, T, H, d_k = q.shape
+    else:
+        T, H, d_k = q.shape
+        B = cu_seqlens.numel() - 1
+    return int(B), int(T), int(H), int(d_k), int(v.shape[-1])
+
+
+def _check(ts, dtype, device_type):
+    for name, t, dt in ts:
+        if t is None:
+            continue
+        if not t.is_contiguous():
+            raise ValueError(f"{name} must be contiguous")
+        if t.dtype != dt:
+            raise ValueError(f"{name} must be {dt}, got {t.dtype}")
+        if t.device.type != device_type:
+            raise ValueError(f"{name} must live on {device_type}, got {t.device}")
+
+
+def _stream(stream):
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return ctypes.c_void_p(stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream))
+
+
+def _prefill(fn_name, io_dtype, q, k, v, log_alpha, beta, initial_state, out, final_state,
+             cu_seqlens, chunk, stream):
+    f32 = torch.float32
+    _check([("q", q, io_dtype), ("k", k, io_dtype), ("v", v, io_dtype), ("out", out, io_dtype),
+            ("log_alpha", log_alpha, f32), ("beta", beta, f32), ("initial_state", initial_state, f32),
+            ("final_state", final_state, f32), ("cu_seqlens", cu_seqlens, torch.int32)], io_dtype, "cuda")
+    B, T, H, d_k, d_v = _dims(q, v, cu_seqlens)
+    if k.shape != q.shape or v.shape[:-1] != q.shape[:-1] or out.shape != v.shape:
+        raise ValueError("q, k, v, out shapes disagree")
+    if log_alpha.shape != q.shape[:-1] or beta.shape != q.shape[:-1]:
+        raise ValueError("gate shapes disagree with q")
+    for name, s in (("initial_state", initial_state), ("final_state", final_state)):
+        if s is not None and tuple(s.shape) != (B, H, d_k, d_v):
+            raise ValueError(f"{name} must be [B,H,d_k,d_v]")
+    rc = getattr(lib(), fn_name)(_ptr(q), _ptr(k), _ptr(v), _ptr(log_alpha), _ptr(beta), _ptr(initial_state),
+                                 _ptr(out), _ptr(final_state), _ptr(cu_seqlens), B, T, H, d_k, d_v,
+                                 int(chunk), _stream(stream))
+    if rc != 0:
+        raise GdnError(rc, fn_name)
+    return out, final_state
+
+
+def gdn_chunk_prefill(q, k, v, log_alpha, beta, initial_state, out, final_state, cu_seqlens=None,
+                      chunk: int = 64, stream=None):
+    """bf16 q/k/v/out; see ``gdn_chunk_prefill`` in include/gdn.h."""
+    return _prefill("gdn_chunk_prefill", torch.bfloat16, q, k, v, log_alpha, beta, initial_state, out,
+                    final_state, cu_seqlens, chunk, stream)
+
+
+def gdn_chunk_prefill_f32(q, k, v, log_alpha, beta, initial_state, out, final_state, cu_seqlens=None,
+                          chunk: int = 64, stream=None):
+    """fp32 q/k/v/out, fp32 arithmetic; see include/gdn.h."""
+    return _prefill("gdn_chunk_prefill_f32", torch.float32, q, k, v, log_alpha, beta, initial_state, out,
+                    final_state, cu_seqlens, chunk, stream)
+
+
+def gdn_chunk_prefill_bf16_simt(q, k, v, log_alpha, beta, initial_state, out, final_state, cu_seqlens=None,
+                                chunk: int = 64, stream=None):
+    """bf16 q/k/v/out through the fp32-arithmetic kernel; see include/gdn.h."""
+    return _prefill("gdn_chunk_prefill_bf16_simt", torch.bfloat16, q, k, v, log_alpha, beta, initial_state,
+                    out, final_state, cu_seqlens, chunk, stream)
+
+
+def gdn_chunk_prefill_host(q, k, v, log_alpha, beta, initial_state, out, final_state, cu_seqlens,
+                           staging: torch.Tensor, chunk: int = 64, stream=None):
+    """Host (CPU, ideally pinned) tensors in and out; ``staging`` is a CUDA uint8 tensor of at
+    least ``gdn_host_staging_bytes`` bytes.  Work is enqueued on ``stream``; synchronise it before
+    reading ``out``."""
+    f32, bf = torch.float32, torch.bfloat16
+    _check([("q", q, bf), ("k", k, bf), ("v", v, bf), ("out", out, bf), ("log_alpha", log_alpha, f32),
+            ("beta", beta, f32), ("initial_state", initial_state, f32), ("final_state", final_state, f32),
+            ("cu_seqlens", cu_seqlens, torch.int32)], bf, "cpu")
+    if staging.device.type != "cuda" or not staging.is_contiguous():
+        raise ValueError("staging must be a contiguous CUDA tensor")
+    B, T, H, d_k, d_v = _dims(q, v, cu_seqlens)
+    rc = lib().gdn_chunk_prefill_host(_ptr(q), _ptr(k), _ptr(v), _ptr(log_alpha), _ptr(beta),
+                                      _ptr(initial_state), _ptr(out), _ptr(final_state), _ptr(cu_seqlens),
+                                      B, T, H, d_k, d_v, int(chunk), _ptr(staging),
+                                      staging.numel() * staging.element_size(), _stream(stream))
+    if rc != 0:
+        raise GdnError(rc, "gdn_chunk_prefill_host")
+    return out, final_state

@@ -1,0 +1,167 @@
+// C-ABI entry points of libgdn: argument validation and dispatch.  See include/gdn.h.
+
+#include <atomic>
+
+#include "gdn_internal.h"
+
+namespace gdn {
+
+static std::atomic<unsigned long long> g_launches{0};
+void count_launch(int n) { g_launches.fetch_add((unsigned long long)n, std::memory_order_relaxed); }
+
+namespace {
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Checks shared by every prefill entry point.  Returns GDN_OK or the error to report.
+int validate(const PrefillArgs& a, int chunk) {
+    if (!a.q || !a.k || !a.v || !a.log_alpha || !a.beta || !a.out) return GDN_ERR_INVALID_ARG;
+    if (a.B <= 0 || a.T < 0 || a.H <= 0 || a.d_k <= 0 || a.d_v <= 0) return GDN_ERR_INVALID_ARG;
+    if (chunk != kChunk) return GDN_ERR_UNSUPPORTED;
+    const void* ptrs[] = {a.q, a.k, a.v, a.log_alpha, a.beta, a.initial_state, a.out, a.final_state};
+    for (const void* p : ptrs)
+        if (p && !aligned16(p)) return GDN_ERR_UNSUPPORTED;
+    if (a.cu_seqlens && (reinterpret_cast<uintptr_t>(a.cu_seqlens) & 3u)) return GDN_ERR_UNSUPPORTED;
+    return GDN_OK;
+}
+
+PrefillArgs pack(const void* q, const void* k, const void* v, const float* log_alpha, const float* beta,
+                 const float* initial_state, void* out, float* final_state, const int32_t* cu_seqlens,
+                 int B, int T, int H, int d_k, int d_v) {
+    return PrefillArgs{q, k, v, log_alpha, beta, initial_state, out, final_state, cu_seqlens, B, T, H, d_k, d_v};
+}
+
+int dispatch_bf16(const PrefillArgs& a, cudaStream_t stream) {
+    if (tc_supported(a.d_k, a.d_v)) return launch_tc(a, stream);
+    return launch_simt(a, /*io_bf16=*/true, stream);
+}
+
+inline size_t up256(size_t x) { return (x + 255) & ~(size_t)255; }
+
+// Device staging area of the host-buffer entry point: offsets of each tensor.
+struct Staging {
+    size_t q, k, v, a, b, s0, out, sT, cu, total;
+    size_t n_qk, n_v, n_gate, n_state, n_cu;   // byte sizes
+};
+
+bool staging_layout(int B, int T, int H, int d_k, int d_v, bool packed, Staging* L) {
+    if (B <= 0 || T < 0 || H <= 0 || d_k <= 0 || d_v <= 0) return false;
+    const size_t tok = packed ? (size_t)T : (size_t)B * T;
+    L->n_qk = tok * H * d_k * sizeof(__nv_bfloat16);
+    L->n_v = tok * H * d_v * sizeof(__nv_bfloat16);
+    L->n_gate = tok * H * sizeof(float);
+    L->n_state = (size_t)B * H * d_k * d_v * sizeof(float);
+    L->n_cu = (size_t)(B + 1) * sizeof(int32_t);
+    size_t o = 0;
+    L->q = o;   o += up256(L->n_qk);
+    L->k = o;   o += up256(L->n_qk);
+    L->v = o;   o += up256(L->n_v);
+    L->a = o;   o += up256(L->n_gate);
+    L->b = o;   o += up256(L->n_gate);
+    L->s0 = o;  o += up256(L->n_state);
+    L->out = o; o += up256(L->n_v);
+    L->sT = o;  o += up256(L->n_state);
+    L->cu = o;  o += up256(L->n_cu);
+    L->total = o;
+    return true;
+}
+
+}  // namespace
+}  // namespace gdn
+
+using namespace gdn;
+
+extern "C" {
+
+int gdn_chunk_prefill(const void* q, const void* k, const void* v, const float* log_alpha,
+                      const float* beta, const float* initial_state, void* out, float* final_state,
+                      const int32_t* cu_seqlens, int B, int T, int H, int d_k, int d_v, int chunk,
+                      gdn_stream_t stream) {
+    const PrefillArgs a = pack(q, k, v, log_alpha, beta, initial_state, out, final_state, cu_seqlens, B, T, H, d_k, d_v);
+    if (int rc = validate(a, chunk)) return rc;
+    return dispatch_bf16(a, reinterpret_cast<cudaStream_t>(stream));
+}
+
+int gdn_chunk_prefill_f32(const float* q, const float* k, const float* v, const float* log_alpha,
+                          const float* beta, const float* initial_state, float* out, float* final_state,
+                          const int32_t* cu_seqlens, int B, int T, int H, int d_k, int d_v, int chunk,
+                          gdn_stream_t stream) {
+    const PrefillArgs a = pack(q, k, v, log_alpha, beta, initial_state, out, final_state, cu_seqlens, B, T, H, d_k, d_v);
+    if (int rc = validate(a, chunk)) return rc;
+    return launch_simt(a, /*io_bf16=*/false, reinterpret_cast<cudaStream_t>(stream));
+}
+
+int gdn_chunk_prefill_bf16_simt(const void* q, const void* k, const void* v, const float* log_alpha,
+                                const float* beta, const float* initial_state, void* out, float* final_state,
+                                const int32_t* cu_seqlens, int B, int T, int H, int d_k, int d_v, int chunk,
+                                gdn_stream_t stream) {
+    const PrefillArgs a = pack(q, k, v, log_alpha, beta, initial_state, out, final_state, cu_seqlens, B, T, H, d_k, d_v);
+    if (int rc = validate(a, chunk)) return rc;
+    return launch_simt(a, /*io_bf16=*/true, reinterpret_cast<cudaStream_t>(stream));
+}
+
+size_t gdn_host_staging_bytes(int B, int T, int H, int d_k, int d_v) {
+    Staging L;
+    // The packed and the batched layouts differ only in how many tokens T stands for; the
+    // larger of the two (B*T) always suffices.
+    return staging_layout(B, T, H, d_k, d_v, /*packed=*/false, &L) ? L.total : 0;
+}
+
+int gdn_chunk_prefill_host(const void* q_host, const void* k_host, const void* v_host,
+                           const float* log_alpha_host, const float* beta_host,
+                           const float* initial_state_host, void* out_host, float* final_state_host,
+                           const int32_t* cu_seqlens_host, int B, int T, int H, int d_k, int d_v, int chunk,
+                           void* staging_dev, size_t staging_bytes, gdn_stream_t stream_) {
+    if (!q_host || !k_host || !v_host || !log_alpha_host || !beta_host || !out_host || !staging_dev)
+        return GDN_ERR_INVALID_ARG;
+    Staging L;
+    if (!staging_layout(B, T, H, d_k, d_v, cu_seqlens_host != nullptr, &L)) return GDN_ERR_INVALID_ARG;
+    if (chunk != kChunk) return GDN_ERR_UNSUPPORTED;
+    if (reinterpret_cast<uintptr_t>(staging_dev) & 255u) return GDN_ERR_UNSUPPORTED;
+    if (staging_bytes < L.total) return GDN_ERR_WORKSPACE;
+    if (cu_seqlens_host) {
+        if (cu_seqlens_host[0] != 0 || cu_seqlens_host[B] != T) return GDN_ERR_INVALID_ARG;
+        for (int n = 0; n < B; ++n)
+            if (cu_seqlens_host[n + 1] < cu_seqlens_host[n]) return GDN_ERR_INVALID_ARG;
+    }
+    cudaStream_t stream = reinterpret_cast<cudaStream_t>(stream_);
+    char* base = static_cast<char*>(staging_dev);
+    auto h2d = [&](size_t off, const void* src, size_t bytes) {
+        return bytes == 0 || cudaMemcpyAsync(base + off, src, bytes, cudaMemcpyHostToDevice, stream) == cudaSuccess;
+    };
+    bool ok = h2d(L.q, q_host, L.n_qk) && h2d(L.k, k_host, L.n_qk) && h2d(L.v, v_host, L.n_v) &&
+              h2d(L.a, log_alpha_host, L.n_gate) && h2d(L.b, beta_host, L.n_gate);
+    if (ok && initial_state_host) ok = h2d(L.s0, initial_state_host, L.n_state);
+    if (ok && cu_seqlens_host) ok = h2d(L.cu, cu_seqlens_host, L.n_cu);
+    if (!ok) return GDN_ERR_CUDA;
+    const PrefillArgs a = pack(base + L.q, base + L.k, base + L.v, reinterpret_cast<const float*>(base + L.a),
+                               reinterpret_cast<const float*>(base + L.b),
+                               initial_state_host ? reinterpret_cast<const float*>(base + L.s0) : nullptr,
+                               base + L.out, final_state_host ? reinterpret_cast<float*>(base + L.sT) : nullptr,
+                               cu_seqlens_host ? reinterpret_cast<const int32_t*>(base + L.cu) : nullptr,
+                               B, T, H, d_k, d_v);
+    if (int rc = validate(a, chunk)) return rc;
+    if (int rc = dispatch_bf16(a, stream)) return rc;
+    if (L.n_v && cudaMemcpyAsync(out_host, base + L.out, L.n_v, cudaMemcpyDeviceToHost, stream) != cudaSuccess)
+        return GDN_ERR_CUDA;
+    if (final_state_host &&
+        cudaMemcpyAsync(final_state_host, base + L.sT, L.n_state, cudaMemcpyDeviceToHost, stream) != cudaSuccess)
+        return GDN_ERR_CUDA;
+    return GDN_OK;
+}
+
+unsigned long long gdn_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+const char* gdn_status_string(int status) {
+    switch (status) {
+        case GDN_OK: return "ok";
+        case GDN_ERR_INVALID_ARG: return "invalid argument";
+        case GDN_ERR_UNSUPPORTED: return "unsupported size, chunk or alignment";
+        case GDN_ERR_WORKSPACE: return "caller-provided scratch too small";
+        case GDN_ERR_CUDA: return "CUDA call or launch failed";
+        case GDN_ERR_TIMEOUT: return "bounded device-side wait expired";
+        default: return "unknown status";
+    }
+}
+
+}  // extern "C"

@@ -1,0 +1,38 @@
+// Internal declarations shared by the translation units of libgdn (not installed).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+
+#include "gdn.h"
+
+namespace gdn {
+
+constexpr int kChunk = 64;
+
+// One prefill call, device pointers.  io_bf16 selects the storage type of q/k/v/out.
+struct PrefillArgs {
+    const void* q;
+    const void* k;
+    const void* v;
+    const float* log_alpha;
+    const float* beta;
+    const float* initial_state;
+    void* out;
+    float* final_state;
+    const int32_t* cu_seqlens;
+    int B, T, H, d_k, d_v;
+};
+
+// fp32-arithmetic kernel (plain FMA); TIO = float or __nv_bfloat16 storage.
+int launch_simt(const PrefillArgs& a, bool io_bf16, cudaStream_t stream);
+bool simt_supported(int d_k, int d_v);
+
+// Tensor-core (tcgen05) kernel for bf16 storage.
+int launch_tc(const PrefillArgs& a, cudaStream_t stream);
+bool tc_supported(int d_k, int d_v);
+
+void count_launch(int n = 1);
+
+}  // namespace gdn

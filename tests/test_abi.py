@@ -1,0 +1,64 @@
+"""The C-ABI library builds, loads without a GPU, and exports every symbol its header declares."""
+import ctypes
+import os
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def libpath():
+    from paper_2607_14568_b200 import build
+    return build.build()
+
+
+def declared_functions():
+    names = []
+    for fn in sorted(os.listdir(os.path.join(ROOT, "include"))):
+        if not fn.endswith(".h"):
+            continue
+        text = open(os.path.join(ROOT, "include", fn)).read()
+        text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+        names += re.findall(r"\b(gdn_[a-z0-9_]+)\s*\(", text)
+    return sorted(set(names))
+
+
+def test_header_symbols_exported(libpath):
+    names = declared_functions()
+    assert "gdn_chunk_prefill" in names and len(names) >= 6
+    lib = ctypes.CDLL(libpath)
+    for n in names:
+        assert hasattr(lib, n), f"{n} declared in include/ but not exported"
+
+
+def test_binding_has_the_same_names(libpath):
+    import paper_2607_14568_b200 as gdn
+    for n in declared_functions():
+        assert hasattr(gdn, n), f"binding lacks {n}"
+    assert gdn.gdn_status_string(0) == "ok" and gdn.gdn_status_string(5)
+    assert gdn.gdn_host_staging_bytes(1, 64, 1, 128, 128) > 0
+    assert gdn.gdn_host_staging_bytes(0, 64, 1, 128, 128) == 0
+
+
+def test_host_entry_rejects_bad_arguments_without_a_gpu(libpath):
+    """Argument checks of the host-buffer entry point run before any CUDA call."""
+    import numpy as np
+    lib = ctypes.CDLL(libpath)
+    lib.gdn_chunk_prefill_host.restype = ctypes.c_int
+    buf = np.zeros(64 * 128, dtype=np.uint16)
+    p = buf.ctypes.data_as(ctypes.c_void_p)
+    vp = ctypes.c_void_p
+    # NULL staging -> invalid argument
+    rc = lib.gdn_chunk_prefill_host(p, p, p, p, p, None, p, None, None, 1, 64, 1, 128, 128, 64, None,
+                                    ctypes.c_size_t(0), None)
+    assert rc == 1
+    # staging too small -> workspace error (pointer is never dereferenced)
+    rc = lib.gdn_chunk_prefill_host(p, p, p, p, p, None, p, None, None, 1, 64, 1, 128, 128, 64, vp(256),
+                                    ctypes.c_size_t(16), None)
+    assert rc == 3
+    cu = np.array([0, 70], dtype=np.int32)
+    rc = lib.gdn_chunk_prefill_host(p, p, p, p, p, None, p, None, cu.ctypes.data_as(vp), 1, 64, 1, 128, 128, 64,
+                                    vp(256), ctypes.c_size_t(1 << 30), None)
+    assert rc == 1   # cu_seqlens[B] != T

@@ -1,0 +1,207 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the fp64 oracle on
+the same seeded inputs, element by element."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2607_14568_b200 as gdn
+from workloads import chain_inputs, get_config, make_inputs, widen
+
+import oracle
+from gdn_testlib import (BF16_MAX_ABS, BF16_REL_L2, F32_REL_L2, assert_close, f64, run_lib, run_oracle,
+                         to_device)
+
+pytestmark = pytest.mark.gpu
+
+BF16_FNS = {"main": gdn.gdn_chunk_prefill, "simt": gdn.gdn_chunk_prefill_bf16_simt}
+
+
+def check_bf16(x, fn, what):
+    d = to_device(x)
+    out, fin = run_lib(fn, d)
+    o_ref, f_ref = run_oracle(x)
+    r1 = assert_close(f64(out), o_ref, BF16_REL_L2, BF16_MAX_ABS, what + " out")
+    r2 = assert_close(f64(fin), f_ref, BF16_REL_L2, BF16_MAX_ABS, what + " final_state")
+    return r1, r2
+
+
+# ---- configuration 1: fp32 path, whole tensor ------------------------------------------------
+def test_tiny_f32():
+    x = make_inputs(get_config("tiny"))
+    d = to_device(x)
+    out, fin = run_lib(gdn.gdn_chunk_prefill_f32, d)
+    o_ref, f_ref = run_oracle(x)
+    assert_close(f64(out), o_ref, F32_REL_L2, None, "tiny out")
+    assert_close(f64(fin), f_ref, F32_REL_L2, None, "tiny final_state")
+
+
+@pytest.mark.parametrize("T,H,dk,dv", [(1, 1, 32, 32), (63, 2, 64, 96), (65, 1, 128, 32), (200, 3, 96, 64),
+                                       (333, 2, 128, 128)])
+def test_f32_ragged_shapes(T, H, dk, dv):
+    cfg = get_config("tiny", T=T, H=H, d_k=dk, d_v=dv, init_std=0.5, seed=100 + T)
+    x = make_inputs(cfg)
+    d = to_device(x)
+    out, fin = run_lib(gdn.gdn_chunk_prefill_f32, d)
+    o_ref, f_ref = run_oracle(x)
+    assert_close(f64(out), o_ref, F32_REL_L2, None, "out")
+    assert_close(f64(fin), f_ref, F32_REL_L2, None, "final_state")
+
+
+def test_f32_packed_with_empty_sequence_and_aliasing():
+    cfg = get_config("tiny", B=4, H=2, d_k=64, d_v=64, lengths=(70, 0, 129, 64), init_std=0.3, seed=7)
+    x = make_inputs(cfg)
+    d = to_device(x)
+    s0 = d["initial_state"].clone()
+    d["final_state"] = d["initial_state"]            # in-place state update is allowed
+    out, fin = run_lib(gdn.gdn_chunk_prefill_f32, d)
+    o_ref, f_ref = run_oracle(x)
+    assert_close(f64(out), o_ref, F32_REL_L2, None, "out")
+    assert_close(f64(fin), f_ref, F32_REL_L2, None, "final_state")
+    assert torch.equal(fin[1], s0[1])                 # the empty sequence passes its state through
+
+
+def test_f32_null_states_and_split_invariance():
+    cfg = get_config("tiny", T=300, H=2, seed=11)
+    x = make_inputs(cfg)
+    d = to_device(x)
+    d["final_state"] = None
+    out_a, _ = run_lib(gdn.gdn_chunk_prefill_f32, d)
+    o_ref, _ = run_oracle(x)
+    assert_close(f64(out_a), o_ref, F32_REL_L2, None, "out without states")
+    # prefix / suffix with the state handed over == one call
+    T1 = 130
+    parts = []
+    state = None
+    for sl in (slice(0, T1), slice(T1, 300)):
+        dd = {k: (v[:, sl].contiguous() if k in ("q", "k", "v", "log_alpha", "beta") else None)
+              for k, v in d.items() if k in ("q", "k", "v", "log_alpha", "beta")}
+        dd.update(initial_state=state, cu_seqlens=None, out=torch.empty_like(dd["v"]),
+                  final_state=torch.empty((1, 2, 64, 64), device="cuda"))
+        o, state = run_lib(gdn.gdn_chunk_prefill_f32, dd)
+        parts.append(o)
+    assert_close(f64(torch.cat(parts, 1)), o_ref, F32_REL_L2, None, "split out")
+
+
+# ---- bf16 storage, reduced shapes that still span several tiles and a ragged tail ---------------
+@pytest.mark.parametrize("impl", ["main", "simt"])
+@pytest.mark.parametrize("T,H,dv,init", [(64, 1, 128, 0.0), (200, 2, 128, 0.02), (1000, 2, 128, 0.02),
+                                         (130, 2, 256, 0.0), (1, 1, 128, 0.02)])
+def test_bf16_reduced(impl, T, H, dv, init):
+    cfg = get_config("long", T=T, H=H, d_v=dv, init_std=init, seed=20 + T)
+    check_bf16(make_inputs(cfg), BF16_FNS[impl], f"{impl} T={T}")
+
+
+@pytest.mark.parametrize("impl", ["main", "simt"])
+def test_bf16_packed_ragged(impl):
+    cfg = get_config("serving", B=5, H=2, lengths=(257, 64, 0, 1, 700), seed=31)
+    x = make_inputs(cfg)
+    (r, _), _ = check_bf16(x, BF16_FNS[impl], impl + " packed")
+    # each sequence alone gives the same rows
+    d = to_device(x)
+    out, fin = run_lib(BF16_FNS[impl], d)
+    cu = x.cu_seqlens
+    for n in (0, 4):
+        a, b = int(cu[n]), int(cu[n + 1])
+        dd = dict(q=d["q"][None, a:b].contiguous(), k=d["k"][None, a:b].contiguous(),
+                  v=d["v"][None, a:b].contiguous(), log_alpha=d["log_alpha"][None, a:b].contiguous(),
+                  beta=d["beta"][None, a:b].contiguous(), initial_state=d["initial_state"][n:n + 1].contiguous(),
+                  cu_seqlens=None)
+        dd["out"] = torch.empty_like(dd["v"])
+        dd["final_state"] = torch.empty_like(dd["initial_state"])
+        o1, f1 = run_lib(BF16_FNS[impl], dd)
+        assert torch.equal(o1[0], out[a:b]) and torch.equal(f1[0], fin[n])
+
+
+def test_bf16_special_cases():
+    """beta = 0 gives pure decay of the initial state; identity padding changes nothing."""
+    cfg = get_config("long", T=192, H=2, seed=41)
+    x = make_inputs(cfg)
+    x.beta[:] = 0.0
+    d = to_device(x)
+    out, fin = run_lib(gdn.gdn_chunk_prefill, d)
+    G = np.exp(np.cumsum(x.log_alpha.astype(np.float64), axis=1))
+    want = G[..., None] * np.einsum("bhmj,bthm->bthj", x.initial_state.astype(np.float64), widen(x.q))
+    assert_close(f64(out), want, BF16_REL_L2, BF16_MAX_ABS, "pure decay out")
+    assert_close(f64(fin), G[:, -1][..., None, None] * x.initial_state, BF16_REL_L2, BF16_MAX_ABS, "pure decay state")
+
+
+def test_deterministic():
+    x = make_inputs(get_config("short", T=640, H=4))
+    d = to_device(x)
+    o1, f1 = run_lib(gdn.gdn_chunk_prefill, d)
+    o1, f1 = o1.clone(), f1.clone()
+    o2, f2 = run_lib(gdn.gdn_chunk_prefill, d)
+    assert torch.equal(o1, o2) and torch.equal(f1, f2)
+
+
+# ---- the benchmark configurations at full size ----------------------------------------------------
+@pytest.mark.parametrize("name", ["short", "long", "serving"])
+def test_bf16_full_configs(name):
+    x = make_inputs(get_config(name))
+    (ro, mo), (rs, ms) = check_bf16(x, gdn.gdn_chunk_prefill, name)
+    print(f"\n{name}: out rel-L2 {ro:.2e} max-abs {mo:.2e}; state rel-L2 {rs:.2e} max-abs {ms:.2e}")
+
+
+def test_bf16_large_sampled_chains():
+    """Configuration 'large' (B=4, T=32768, H=32, d_v=256) at full size; the oracle checks a seeded
+    sample of whole (sequence, head) chains (heads are independent, so each checked chain is
+    checked completely) and every other chain is checked for finiteness."""
+    cfg = get_config("large")
+    x = make_inputs(cfg, threads=16)
+    d = to_device(x)
+    out, fin = run_lib(gdn.gdn_chunk_prefill, d)
+    assert bool(torch.isfinite(out).all()) and bool(torch.isfinite(fin).all())
+    rng = np.random.default_rng(5)
+    chains = {(0, 0), (cfg.B - 1, cfg.H - 1)} | {(int(rng.integers(cfg.B)), int(rng.integers(cfg.H))) for _ in range(4)}
+    for n, h in sorted(chains):
+        c = chain_inputs(cfg, n, h)
+        o_ref, f_ref = oracle.sequential(widen(c["q"])[None, :, None], widen(c["k"])[None, :, None],
+                                         widen(c["v"])[None, :, None], c["log_alpha"][None, :, None],
+                                         c["beta"][None, :, None], None)
+        assert_close(f64(out[n, :, h]), o_ref[0, :, 0], BF16_REL_L2, BF16_MAX_ABS, f"large chain {(n, h)} out")
+        assert_close(f64(fin[n, h]), f_ref[0, 0], BF16_REL_L2, BF16_MAX_ABS, f"large chain {(n, h)} state")
+
+
+# ---- host-buffer entry point ------------------------------------------------------------------------
+def test_host_entry_matches_device_entry():
+    cfg = get_config("serving", B=3, H=2, lengths=(300, 64, 77), seed=51)
+    x = make_inputs(cfg)
+    d = to_device(x)
+    out, fin = run_lib(gdn.gdn_chunk_prefill, d)
+    h = to_device(x, device="cpu")
+    h = {k: (v.pin_memory() if v is not None else None) for k, v in h.items()}
+    nbytes = gdn.gdn_host_staging_bytes(cfg.B, x.T_arg, cfg.H, cfg.d_k, cfg.d_v)
+    staging = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+    o2, f2 = gdn.gdn_chunk_prefill_host(h["q"], h["k"], h["v"], h["log_alpha"], h["beta"], h["initial_state"],
+                                        h["out"], h["final_state"], h["cu_seqlens"], staging)
+    torch.cuda.synchronize()
+    assert torch.equal(o2, out.cpu()) and torch.equal(f2, fin.cpu())
+    with pytest.raises(gdn.GdnError) as e:
+        gdn.gdn_chunk_prefill_host(h["q"], h["k"], h["v"], h["log_alpha"], h["beta"], h["initial_state"],
+                                   h["out"], h["final_state"], h["cu_seqlens"], staging[:1024])
+    assert e.value.status == 3
+
+
+# ---- error behaviour ---------------------------------------------------------------------------------
+def test_error_codes():
+    x = make_inputs(get_config("long", T=64, H=1))
+    d = to_device(x)
+    n0 = gdn.gdn_launch_count()
+    with pytest.raises(gdn.GdnError) as e:
+        run_lib(gdn.gdn_chunk_prefill, d, chunk=32)
+    assert e.value.status == 2
+    L = gdn.lib()
+    args = [d["q"].data_ptr(), d["k"].data_ptr(), d["v"].data_ptr(), d["log_alpha"].data_ptr(), d["beta"].data_ptr(),
+            None, d["out"].data_ptr(), None, None, 1, 64, 1, 128, 128, 64, None]
+    bad = list(args); bad[0] = None
+    assert L.gdn_chunk_prefill(*bad) == 1
+    bad = list(args); bad[9] = 0
+    assert L.gdn_chunk_prefill(*bad) == 1
+    bad = list(args); bad[1] = d["k"].data_ptr() + 2
+    assert L.gdn_chunk_prefill(*bad) == 2
+    bad = list(args); bad[12] = 100
+    assert L.gdn_chunk_prefill(*bad) == 2
+    assert gdn.gdn_launch_count() == n0              # nothing was launched for any of these
+    assert L.gdn_chunk_prefill(*args) == 0
+    torch.cuda.synchronize()
+    assert gdn.gdn_launch_count() > n0
