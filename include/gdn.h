@@ -124,6 +124,14 @@ int gdn_chunk_prefill_host(const void* q_host, const void* k_host, const void* v
 /* Bytes of device staging gdn_chunk_prefill_host needs for these sizes (0 on bad sizes). */
 size_t gdn_host_staging_bytes(int B, int T, int H, int d_k, int d_v);
 
+/*
+ * Waits for the device to finish (cudaDeviceSynchronize) and returns the status word of
+ * the kernels: GDN_OK, or GDN_ERR_TIMEOUT if a bounded device-side wait (on a TMA copy,
+ * a tensor-core completion or another warp role) ever expired, in which case the outputs
+ * of that call are undefined.  GDN_ERR_CUDA if the device reports an error.
+ */
+int gdn_query_status(void);
+
 /* Number of kernels this library has launched in this process so far. */
 unsigned long long gdn_launch_count(void);
 

@@ -45,6 +45,10 @@ def lib():
         L.gdn_chunk_prefill_host.restype = i
         L.gdn_host_staging_bytes.argtypes = [i] * 5
         L.gdn_host_staging_bytes.restype = sz
+        L.gdn_query_status.argtypes = []
+        L.gdn_query_status.restype = i
+        L.gdn_debug_set_dump.argtypes = [vp]
+        L.gdn_debug_set_dump.restype = None
         L.gdn_launch_count.argtypes = []
         L.gdn_launch_count.restype = ctypes.c_ulonglong
         L.gdn_status_string.argtypes = [i]
@@ -55,6 +59,11 @@ def lib():
 
 def gdn_status_string(status: int) -> str:
     return lib().gdn_status_string(int(status)).decode()
+
+
+def gdn_query_status() -> int:
+    """Synchronises the device and returns the kernels' status word (0 = ok)."""
+    return int(lib().gdn_query_status())
 
 
 def gdn_launch_count() -> int:

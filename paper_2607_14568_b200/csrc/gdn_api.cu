@@ -150,6 +150,11 @@ int gdn_chunk_prefill_host(const void* q_host, const void* k_host, const void* v
     return GDN_OK;
 }
 
+int gdn_query_status(void) { return tc_query_status(); }
+
+// Not part of the public header: lets the tests capture per-stage intermediates.
+void gdn_debug_set_dump(float* device_buffer) { tc_set_debug_dump(device_buffer); }
+
 unsigned long long gdn_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
 const char* gdn_status_string(int status) {

@@ -32,6 +32,8 @@ bool simt_supported(int d_k, int d_v);
 // Tensor-core (tcgen05) kernel for bf16 storage.
 int launch_tc(const PrefillArgs& a, cudaStream_t stream);
 bool tc_supported(int d_k, int d_v);
+int tc_query_status();               // synchronises the device, returns the kernels' status word
+void tc_set_debug_dump(float* p);    // tests only: stage dump of chunk 0 of CTA (0,0,0)
 
 void count_launch(int n = 1);
 
