@@ -69,7 +69,11 @@ constexpr uint32_t SM_T1 = SM_P + 2 * 8192;         // (T diag(b e^g))^T [64 i][
 constexpr uint32_t SM_T2 = SM_T1 + 8192;            // (T diag(b))^T
 constexpr uint32_t SM_A = SM_T2 + 8192;             // fp32 A [64][68]
 constexpr uint32_t LDA = 68;
-constexpr uint32_t SM_GATES = SM_A + 64 * LDA * 4;  // 4 x {g, beta, e^g, e^{gC-g}, e^{gC}}
+constexpr uint32_t SM_TF = SM_A + 64 * LDA * 4;     // fp32 T [64][68]
+constexpr uint32_t SM_Y = SM_TF + 64 * LDA * 4;     // fp32 scratch of the blocked solve [32][36]
+constexpr uint32_t LDY = 36;
+constexpr uint32_t SM_OST = SM_Y + 32 * LDY * 4;    // bf16 output staging [64][128]
+constexpr uint32_t SM_GATES = SM_OST + 64 * 128 * 2;  // 4 x {g log2e, beta, e^g, e^{gC-g}, e^{gC}}
 constexpr uint32_t GATE_FLOATS = 320;
 constexpr uint32_t SM_BARS = SM_GATES + 4 * GATE_FLOATS * 4;
 constexpr uint32_t SM_MISC = SM_BARS + 32 * 8;      // tmem base, abort flag
@@ -78,7 +82,8 @@ constexpr uint32_t SMEM_BYTES = SM_TOTAL + 1024;    // slack for the manual 1024
 
 enum Bar : uint32_t {
     B_FULL0 = 0, B_FULL1, B_FREE0, B_FREE1, B_G, B_W, B_V, B_S, B_O,
-    B_TREADY, B_WREADY0, B_WREADY1, B_SREADY, B_VREADY, B_OFREE, B_COUNT
+    B_TREADY, B_WREADY0, B_WREADY1, B_SREADY, B_VREADY, B_OFREE,
+    B_GREADY0, B_GREADY1, B_GREADY2, B_GREADY3, B_GFREE0, B_GFREE1, B_GFREE2, B_GFREE3, B_COUNT
 };
 
 struct TcParams {
@@ -103,11 +108,10 @@ __device__ __forceinline__ void wait(const Cta& cta, uint32_t bar_idx, uint32_t 
     const uint32_t bar = cta.bar(bar_idx);
     if (mbar_try_wait(bar, parity)) return;
     const unsigned long long t0 = globaltimer_ns();
-    uint32_t spins = 0;
     while (true) {
-        if (mbar_try_wait(bar, parity)) return;
+        if (mbar_try_wait_suspend(bar, parity, 100000u)) return;
         if (*cta.abort_flag) return;
-        if ((++spins & 0x3FF) == 0 && globaltimer_ns() - t0 > TIMEOUT_NS) {
+        if (globaltimer_ns() - t0 > TIMEOUT_NS) {
             *cta.abort_flag = 1;
             atomicCAS(&g_tc_status, 0, (int)GDN_ERR_TIMEOUT);
             return;
@@ -196,6 +200,8 @@ gdn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
     uint8_t* sm = smem_raw + (cta.base - smem_u32(smem_raw));
     float* sA = reinterpret_cast<float*>(sm + SM_A);
     float* sGates = reinterpret_cast<float*>(sm + SM_GATES);
+    float* sTf = reinterpret_cast<float*>(sm + SM_TF);
+    float* sY = reinterpret_cast<float*>(sm + SM_Y);
     volatile uint32_t* sMisc = reinterpret_cast<volatile uint32_t*>(sm + SM_MISC);
     cta.abort_flag = reinterpret_cast<volatile int*>(sm + SM_MISC + 4);
 
@@ -215,6 +221,7 @@ gdn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
         mbar_init(cta.bar(B_S), 1); mbar_init(cta.bar(B_O), 1);
         mbar_init(cta.bar(B_TREADY), 128); mbar_init(cta.bar(B_WREADY0), 128); mbar_init(cta.bar(B_WREADY1), 128);
         mbar_init(cta.bar(B_SREADY), 128); mbar_init(cta.bar(B_VREADY), 128); mbar_init(cta.bar(B_OFREE), 128);
+        for (uint32_t i = 0; i < 4; ++i) { mbar_init(cta.bar(B_GREADY0 + i), 32); mbar_init(cta.bar(B_GFREE0 + i), 128); }
         sMisc[1] = 0;   // abort flag
         fence_mbar_init();
     }
@@ -229,6 +236,12 @@ gdn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
 
     const bool dump = DBG && p.dbg != nullptr && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0;
     const size_t state_off = ((size_t)n * H + h) * DK * dv + (size_t)dvb * DVB;
+    // debug builds: per-role time stamps (ns since kernel start) of the first 16 chunks
+    const unsigned long long t_start = DBG ? globaltimer_ns() : 0ull;
+    auto stamp = [&](int role, int c, int ev) {
+        if (DBG && dump && c < 16)
+            p.dbg[7 * 16384 + (role * 16 + c) * 8 + ev] = (float)(globaltimer_ns() - t_start);
+    };
 
     if (warp < 4) {
         // =============================== chain warpgroup ===============================
@@ -260,6 +273,7 @@ gdn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
             // ---- v_new^T = U^T - S^T W^T is in TM_DV ----
             wait(cta, B_V, c & 1);
             tc_fence_after_sync();
+            if (tid == 0) stamp(0, c, 0);
 #pragma unroll
             for (int hh = 0; hh < 2; ++hh) {
                 uint32_t x[32];
@@ -282,9 +296,11 @@ gdn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
             tmem_wait_st();
             tc_fence_before_sync();
             mbar_arrive(cta.bar(B_VREADY));
+            if (tid == 0) stamp(0, c, 1);
             // ---- S^T <- e^{gC} S^T + (v e^{gC-g})^T K ----
             wait(cta, B_S, c & 1);
             tc_fence_after_sync();
+            if (tid == 0) stamp(0, c, 2);
             const float gamma = gates[256];
 #pragma unroll
             for (int q = 0; q < 4; ++q) {
@@ -304,6 +320,7 @@ gdn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
             tmem_wait_st();
             tc_fence_before_sync();
             mbar_arrive(cta.bar(B_SREADY));
+            if (tid == 0) stamp(0, c, 3);
         }
         if (p.sT) {
 #pragma unroll
@@ -314,103 +331,192 @@ gdn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
         const int tp = tid - 128, wp = tp >> 5;
         const uint32_t lane_base = (uint32_t)(wp * 32) << 16;
         for (int c = 0; c < nchunks; ++c) {
-            const int R = min(C, len - c * C);
             const uint32_t buf = c & 1;
-            float* gates = sGates + (c & 3) * GATE_FLOATS;
-            // ---- step a: chunk-local cumulative log gate ----
-            if (wp == 0) {
-                const int r0 = lane, r1 = lane + 32;
-                float x = 0.f, y = 0.f, b0 = 0.f, b1 = 0.f;
-                if (r0 < R) { const size_t o = (size_t)(tok0 + c * C + r0) * H + h; x = __ldg(p.a + o); b0 = __ldg(p.beta + o); }
-                if (r1 < R) { const size_t o = (size_t)(tok0 + c * C + r1) * H + h; y = __ldg(p.a + o); b1 = __ldg(p.beta + o); }
-#pragma unroll
-                for (int d = 1; d < 32; d <<= 1) {
-                    const float xu = __shfl_up_sync(0xffffffffu, x, d);
-                    const float yu = __shfl_up_sync(0xffffffffu, y, d);
-                    if (lane >= d) { x += xu; y += yu; }
-                }
-                y += __shfl_sync(0xffffffffu, x, 31);
-                const float gC = __shfl_sync(0xffffffffu, y, 31);
-                gates[r0] = x; gates[r1] = y;
-                gates[64 + r0] = b0; gates[64 + r1] = b1;
-                gates[128 + r0] = ex2(x * LOG2E); gates[128 + r1] = ex2(y * LOG2E);
-                gates[192 + r0] = ex2((gC - x) * LOG2E); gates[192 + r1] = ex2((gC - y) * LOG2E);
-                if (lane == 0) gates[256] = ex2(gC * LOG2E);
-            }
-            named_bar_sync(1, 128);
+            const float* gates = sGates + (c & 3) * GATE_FLOATS;
+            if (tp == 0) stamp(1, c, 0);
+            wait(cta, B_GREADY0 + (c & 3), (c >> 2) & 1);      // step a runs ahead in its own warp
+            if (tp == 0) stamp(1, c, 1);
             // ---- step b1: decay masks on G = [K;Q] K^T ----
             wait(cta, B_G, c & 1);
             tc_fence_after_sync();
+            if (tp == 0) stamp(1, c, 2);
             {
-                uint32_t x[64];
-                {
-                    uint32_t lo[32], hi[32];
-                    tmem_ld32(cta.tmem + lane_base + TM_GW, lo);
-                    tmem_ld32(cta.tmem + lane_base + TM_GW + 32, hi);
-                    tmem_wait_ld();
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) { x[i] = lo[i]; x[32 + i] = hi[i]; }
-                }
-                if (dump && c == 0)
-#pragma unroll
-                    for (int i = 0; i < 64; ++i) p.dbg[tp * 64 + i] = __uint_as_float(x[i]);
                 const int r = tp & 63;
-                const float gr = gates[r] * LOG2E;
-                if (tp < 64) {
-                    const float br = gates[64 + r];
+                const float gr = gates[r];
+                const float br = gates[64 + r];
+                const bool is_a = tp < 64;                 // warps 0,1: A rows; warps 2,3: P rows
+                const int rmax = 32 * (wp & 1) + 31;       // largest row held by this warp
+                const uint32_t pimg = cta.base + SM_P + buf * 8192;
 #pragma unroll
-                    for (int i4 = 0; i4 < 16; ++i4) {
-                        float o[4];
+                for (int hh = 0; hh < 2; ++hh) {
+                    if (32 * hh <= rmax) {
+                        uint32_t x[32];
+                        tmem_ld32(cta.tmem + lane_base + TM_GW + 32 * hh, x);
+                        tmem_wait_ld();
+                        if (dump && c == 0)
 #pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            const int i = 4 * i4 + e;
-                            const float dec = ex2(gr - gates[i] * LOG2E);
-                            o[e] = (i < r) ? br * dec * __uint_as_float(x[i]) : 0.f;
+                            for (int i = 0; i < 32; ++i) p.dbg[tp * 64 + 32 * hh + i] = __uint_as_float(x[i]);
+                        float y[32];
+#pragma unroll
+                        for (int i4 = 0; i4 < 8; ++i4) {
+                            const float4 gi = *reinterpret_cast<const float4*>(gates + 32 * hh + 4 * i4);
+                            y[4 * i4 + 0] = ex2(gr - gi.x) * __uint_as_float(x[4 * i4 + 0]);
+                            y[4 * i4 + 1] = ex2(gr - gi.y) * __uint_as_float(x[4 * i4 + 1]);
+                            y[4 * i4 + 2] = ex2(gr - gi.z) * __uint_as_float(x[4 * i4 + 2]);
+                            y[4 * i4 + 3] = ex2(gr - gi.w) * __uint_as_float(x[4 * i4 + 3]);
                         }
-                        st_shared_f4(cta.base + SM_A + (r * LDA + 4 * i4) * 4, o[0], o[1], o[2], o[3]);
-                    }
-                } else {
-                    const uint32_t pimg = cta.base + SM_P + buf * 8192;
+                        if (is_a) {
 #pragma unroll
-                    for (int ch = 0; ch < 8; ++ch) {
-                        uint32_t pk[4];
+                            for (int i4 = 0; i4 < 8; ++i4) {
+                                float o[4];
 #pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            const int i0 = 8 * ch + 2 * e, i1 = i0 + 1;
-                            const float d0 = ex2(gr - gates[i0] * LOG2E), d1 = ex2(gr - gates[i1] * LOG2E);
-                            const float p0 = (i0 <= r) ? d0 * __uint_as_float(x[i0]) : 0.f;
-                            const float p1 = (i1 <= r) ? d1 * __uint_as_float(x[i1]) : 0.f;
-                            pk[e] = pack_bf16(p0, p1);
+                                for (int e = 0; e < 4; ++e) {
+                                    const int i = 32 * hh + 4 * i4 + e;
+                                    o[e] = (i < r) ? br * y[4 * i4 + e] : 0.f;
+                                }
+                                st_shared_f4(cta.base + SM_A + (r * LDA + 32 * hh + 4 * i4) * 4, o[0], o[1], o[2], o[3]);
+                            }
+                        } else {
+#pragma unroll
+                            for (int ch = 0; ch < 4; ++ch) {
+                                uint32_t pk[4];
+#pragma unroll
+                                for (int e = 0; e < 4; ++e) {
+                                    const int i0 = 32 * hh + 8 * ch + 2 * e;
+                                    pk[e] = pack_bf16((i0 <= r) ? y[8 * ch + 2 * e] : 0.f,
+                                                      (i0 + 1 <= r) ? y[8 * ch + 2 * e + 1] : 0.f);
+                                }
+                                st_shared_v4(pimg + swz(r, 4 * hh + ch), pk[0], pk[1], pk[2], pk[3]);
+                            }
                         }
-                        st_shared_v4(pimg + swz(r, ch), pk[0], pk[1], pk[2], pk[3]);
+                    } else if (!is_a) {
+#pragma unroll
+                        for (int ch = 0; ch < 4; ++ch) st_shared_v4(pimg + swz(r, 4 * hh + ch), 0u, 0u, 0u, 0u);
                     }
                 }
             }
             named_bar_sync(1, 128);
-            // ---- step b2: forward substitution, column tp of T = (I + A)^{-1} ----
+            if (tp == 0) stamp(1, c, 3);
+            // ---- step b2: T = (I + A)^{-1} by blocked forward substitution (fp32, shared memory) ----
+            // level 0: the four 16x16 diagonal blocks, one column per thread, no barrier inside
             if (tp < 64) {
-                const int cc = tp;
-                float t[64];
+                const int I = tp >> 4, cc = tp & 15;
+                const float* Ab = sA + (16 * I) * LDA + 16 * I;
+                float* Tb = sTf + (16 * I) * LDA + 16 * I;
+                float xs[16];
 #pragma unroll
-                for (int r = 0; r < 64; ++r) {
-                    float acc0 = 0.f, acc1 = 0.f, acc2 = 0.f, acc3 = 0.f;
+                for (int r = 0; r < 16; ++r) {
+                    float acc0 = 0.f, acc1 = 0.f;
 #pragma unroll
                     for (int i4 = 0; i4 < (r + 3) / 4; ++i4) {
-                        const float4 a4 = *reinterpret_cast<const float4*>(sA + r * LDA + 4 * i4);
-                        if (4 * i4 + 0 < r) acc0 = fmaf(a4.x, t[4 * i4 + 0], acc0);
-                        if (4 * i4 + 1 < r) acc1 = fmaf(a4.y, t[4 * i4 + 1], acc1);
-                        if (4 * i4 + 2 < r) acc2 = fmaf(a4.z, t[4 * i4 + 2], acc2);
-                        if (4 * i4 + 3 < r) acc3 = fmaf(a4.w, t[4 * i4 + 3], acc3);
+                        const float4 a4 = *reinterpret_cast<const float4*>(Ab + r * LDA + 4 * i4);
+                        if (4 * i4 + 0 < r) acc0 = fmaf(a4.x, xs[4 * i4 + 0], acc0);
+                        if (4 * i4 + 1 < r) acc1 = fmaf(a4.y, xs[4 * i4 + 1], acc1);
+                        if (4 * i4 + 2 < r) acc0 = fmaf(a4.z, xs[4 * i4 + 2], acc0);
+                        if (4 * i4 + 3 < r) acc1 = fmaf(a4.w, xs[4 * i4 + 3], acc1);
                     }
-                    t[r] = ((r == cc) ? 1.f : 0.f) - ((acc0 + acc1) + (acc2 + acc3));
+                    xs[r] = ((r == cc) ? 1.f : 0.f) - (acc0 + acc1);
+                    Tb[r * LDA + cc] = xs[r];
+                }
+            }
+            named_bar_sync(1, 128);
+            // level 1: 16-blocks (1,0) and (3,2):  T21 = -T22 (A21 T11)
+            {
+                const int pr = tp >> 6, r = (tp >> 2) & 15, cg = tp & 3;
+                const int lo = 32 * pr, hi = lo + 16;
+                float acc[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll 1
+                for (int i4 = 0; i4 < 4; ++i4) {
+                    const float4 a4 = *reinterpret_cast<const float4*>(sA + (hi + r) * LDA + lo + 4 * i4);
+                    const float av[4] = {a4.x, a4.y, a4.z, a4.w};
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const float4 t4 = *reinterpret_cast<const float4*>(sTf + (lo + 4 * i4 + e) * LDA + lo + 4 * cg);
+                        acc[0] = fmaf(av[e], t4.x, acc[0]); acc[1] = fmaf(av[e], t4.y, acc[1]);
+                        acc[2] = fmaf(av[e], t4.z, acc[2]); acc[3] = fmaf(av[e], t4.w, acc[3]);
+                    }
+                }
+                *reinterpret_cast<float4*>(sY + (16 * pr + r) * LDY + 4 * cg) = make_float4(acc[0], acc[1], acc[2], acc[3]);
+                named_bar_sync(1, 128);
+                float t[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll 1
+                for (int i4 = 0; i4 < 4; ++i4) {
+                    const float4 a4 = *reinterpret_cast<const float4*>(sTf + (hi + r) * LDA + hi + 4 * i4);
+                    const float av[4] = {a4.x, a4.y, a4.z, a4.w};
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const float4 y4 = *reinterpret_cast<const float4*>(sY + (16 * pr + 4 * i4 + e) * LDY + 4 * cg);
+                        t[0] = fmaf(av[e], y4.x, t[0]); t[1] = fmaf(av[e], y4.y, t[1]);
+                        t[2] = fmaf(av[e], y4.z, t[2]); t[3] = fmaf(av[e], y4.w, t[3]);
+                    }
+                }
+                *reinterpret_cast<float4*>(sTf + (hi + r) * LDA + lo + 4 * cg) = make_float4(-t[0], -t[1], -t[2], -t[3]);
+                // the not-yet-written upper-right 16-blocks of the two 32-blocks are zero
+                *reinterpret_cast<float4*>(sTf + (lo + r) * LDA + hi + 4 * cg) = make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+            named_bar_sync(1, 128);
+            // level 2: the 32-block (1,0):  T21 = -T22 (A21 T11)
+            {
+                const int r = tp >> 2, cg = tp & 3;
+                float acc[8];
+#pragma unroll
+                for (int e = 0; e < 8; ++e) acc[e] = 0.f;
+#pragma unroll 1
+                for (int i4 = 0; i4 < 8; ++i4) {
+                    const float4 a4 = *reinterpret_cast<const float4*>(sA + (32 + r) * LDA + 4 * i4);
+                    const float av[4] = {a4.x, a4.y, a4.z, a4.w};
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const float* trow = sTf + (4 * i4 + e) * LDA + 8 * cg;
+                        const float4 t0 = *reinterpret_cast<const float4*>(trow);
+                        const float4 t1 = *reinterpret_cast<const float4*>(trow + 4);
+                        acc[0] = fmaf(av[e], t0.x, acc[0]); acc[1] = fmaf(av[e], t0.y, acc[1]);
+                        acc[2] = fmaf(av[e], t0.z, acc[2]); acc[3] = fmaf(av[e], t0.w, acc[3]);
+                        acc[4] = fmaf(av[e], t1.x, acc[4]); acc[5] = fmaf(av[e], t1.y, acc[5]);
+                        acc[6] = fmaf(av[e], t1.z, acc[6]); acc[7] = fmaf(av[e], t1.w, acc[7]);
+                    }
+                }
+                *reinterpret_cast<float4*>(sY + r * LDY + 8 * cg) = make_float4(acc[0], acc[1], acc[2], acc[3]);
+                *reinterpret_cast<float4*>(sY + r * LDY + 8 * cg + 4) = make_float4(acc[4], acc[5], acc[6], acc[7]);
+                named_bar_sync(1, 128);
+                float t[8];
+#pragma unroll
+                for (int e = 0; e < 8; ++e) t[e] = 0.f;
+#pragma unroll 1
+                for (int i4 = 0; i4 < 8; ++i4) {
+                    const float4 a4 = *reinterpret_cast<const float4*>(sTf + (32 + r) * LDA + 32 + 4 * i4);
+                    const float av[4] = {a4.x, a4.y, a4.z, a4.w};
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const float* yrow = sY + (4 * i4 + e) * LDY + 8 * cg;
+                        const float4 y0 = *reinterpret_cast<const float4*>(yrow);
+                        const float4 y1 = *reinterpret_cast<const float4*>(yrow + 4);
+                        t[0] = fmaf(av[e], y0.x, t[0]); t[1] = fmaf(av[e], y0.y, t[1]);
+                        t[2] = fmaf(av[e], y0.z, t[2]); t[3] = fmaf(av[e], y0.w, t[3]);
+                        t[4] = fmaf(av[e], y1.x, t[4]); t[5] = fmaf(av[e], y1.y, t[5]);
+                        t[6] = fmaf(av[e], y1.z, t[6]); t[7] = fmaf(av[e], y1.w, t[7]);
+                    }
+                }
+                *reinterpret_cast<float4*>(sTf + (32 + r) * LDA + 8 * cg) = make_float4(-t[0], -t[1], -t[2], -t[3]);
+                *reinterpret_cast<float4*>(sTf + (32 + r) * LDA + 8 * cg + 4) = make_float4(-t[4], -t[5], -t[6], -t[7]);
+            }
+            named_bar_sync(1, 128);
+            // ---- step b3 operands: rows i of (T diag(b e^g))^T and (T diag(b))^T; thread = (column, half) ----
+            {
+                const int cc = tp & 63, half = tp >> 6;
+                const float b = gates[64 + cc], bg = b * gates[128 + cc];
+                float t[32];
+#pragma unroll
+                for (int i = 0; i < 32; ++i) {
+                    const int r = 32 * half + i;
+                    // rows above the 32-block of this column were never written: they are zero
+                    t[i] = (half == 0 && cc >= 32) ? 0.f : sTf[r * LDA + cc];
                 }
                 if (dump && c == 0)
 #pragma unroll
-                    for (int r = 0; r < 64; ++r) p.dbg[1 * 16384 + r * 64 + cc] = t[r];
-                // step b3 operands: rows i = cc of (T diag(b e^g))^T and (T diag(b))^T
-                const float b = gates[64 + cc], bg = b * gates[128 + cc];
+                    for (int i = 0; i < 32; ++i) p.dbg[1 * 16384 + (32 * half + i) * 64 + cc] = t[i];
 #pragma unroll
-                for (int ch = 0; ch < 8; ++ch) {
+                for (int ch = 0; ch < 4; ++ch) {
                     uint32_t p1[4], p2[4];
 #pragma unroll
                     for (int e = 0; e < 4; ++e) {
@@ -418,16 +524,18 @@ gdn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
                         p1[e] = pack_bf16(t0 * bg, t1 * bg);
                         p2[e] = pack_bf16(t0 * b, t1 * b);
                     }
-                    st_shared_v4(cta.base + SM_T1 + swz(cc, ch), p1[0], p1[1], p1[2], p1[3]);
-                    st_shared_v4(cta.base + SM_T2 + swz(cc, ch), p2[0], p2[1], p2[2], p2[3]);
+                    st_shared_v4(cta.base + SM_T1 + swz(cc, 4 * half + ch), p1[0], p1[1], p1[2], p1[3]);
+                    st_shared_v4(cta.base + SM_T2 + swz(cc, 4 * half + ch), p2[0], p2[1], p2[2], p2[3]);
                 }
             }
             fence_proxy_async_smem();
             tc_fence_before_sync();
+            if (tp == 0) stamp(1, c, 4);
             mbar_arrive(cta.bar(B_TREADY));
             // ---- step b3 result: -W^T from tensor memory to its shared-memory image ----
             wait(cta, B_W, c & 1);
             tc_fence_after_sync();
+            if (tp == 0) stamp(1, c, 5);
             {
                 const uint32_t wimg = cta.base + SM_W + buf * 16384;
 #pragma unroll
@@ -451,18 +559,20 @@ gdn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
             fence_proxy_async_smem();
             tc_fence_before_sync();
             mbar_arrive(cta.bar(B_WREADY0 + buf));
+            if (tp == 0) stamp(1, c, 6);
         }
     } else if (warp < 12) {
         // =============================== epilogue warpgroup ===============================
         setmaxnreg_dec<96>();
         const int j = tid - 256, we = j >> 5;
         const uint32_t lane_base = (uint32_t)(we * 32) << 16;
+        __nv_bfloat16* ost = reinterpret_cast<__nv_bfloat16*>(sm + SM_OST);   // [64 rows][128 columns]
         for (int c = 0; c < nchunks; ++c) {
             const int R = min(C, len - c * C);
             const float* gates = sGates + (c & 3) * GATE_FLOATS;
-            __nv_bfloat16* orow = p.out + ((size_t)(tok0 + c * C) * H + h) * dv + (size_t)dvb * DVB + j;
             wait(cta, B_O, c & 1);
             tc_fence_after_sync();
+            if (j == 0) stamp(2, c, 0);
 #pragma unroll
             for (int hh = 0; hh < 2; ++hh) {
                 uint32_t o1[32], o2[32];
@@ -483,9 +593,25 @@ gdn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
                 for (int i = 0; i < 32; ++i) {
                     const int r = 32 * hh + i;
                     const float o = fmaf(gates[128 + r], __uint_as_float(o1[i]), __uint_as_float(o2[i]));
-                    if (r < R) orow[(size_t)r * H * dv] = __float2bfloat16_rn(o);
+                    ost[r * DVB + j] = __float2bfloat16_rn(o);      // transpose through shared memory
                 }
             }
+            named_bar_sync(2, 128);
+            // coalesced 16-byte stores: 16 threads cover one 256-byte output row
+            {
+                __nv_bfloat16* obase = p.out + ((size_t)(tok0 + c * C) * H + h) * dv + (size_t)dvb * DVB;
+#pragma unroll
+                for (int it = 0; it < 8; ++it) {
+                    const int qd = it * 128 + j, r = qd >> 4, col = (qd & 15) * 8;
+                    if (r < R) {
+                        const uint4 val = *reinterpret_cast<const uint4*>(ost + r * DVB + col);
+                        *reinterpret_cast<uint4*>(obase + (size_t)r * H * dv + col) = val;
+                    }
+                }
+            }
+            named_bar_sync(2, 128);
+            mbar_arrive(cta.bar(B_GFREE0 + (c & 3)));          // last reader of this chunk's gate vectors
+            if (j == 0) stamp(2, c, 1);
         }
     } else {
         // =============================== control warpgroup ===============================
@@ -508,6 +634,7 @@ gdn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
                 wait(cta, B_SREADY, c & 1);
                 wait(cta, B_WREADY0 + buf, par2);
                 tc_fence_after_sync();
+                stamp(3, c, 0);
                 issue_1(cta, buf);
                 mma_commit(cta.bar(B_V));
                 if (c > 0) { wait(cta, B_OFREE, (c - 1) & 1); tc_fence_after_sync(); }
@@ -518,8 +645,10 @@ gdn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
                     issue_G(cta, nb);
                     mma_commit(cta.bar(B_G));
                 }
+                stamp(3, c, 1);
                 wait(cta, B_VREADY, c & 1);
                 tc_fence_after_sync();
+                stamp(3, c, 2);
                 issue_2(cta, buf);
                 mma_commit(cta.bar(B_S));
                 issue_o2(cta, buf);
@@ -528,10 +657,37 @@ gdn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
                 if (c + 1 < nchunks) {
                     wait(cta, B_TREADY, (c + 1) & 1);
                     tc_fence_after_sync();
+                    stamp(3, c, 3);
                     issue_Wt(cta, (c + 1) & 1);
                     mma_commit(cta.bar(B_W));
                     issue_U(cta, (c + 1) & 1);
                 }
+                stamp(3, c, 4);
+            }
+        } else if (warp == 14) {
+            // ---- step a: chunk-local cumulative log gate, up to four chunks ahead ----
+            for (int c = 0; c < nchunks; ++c) {
+                const int R = min(C, len - c * C);
+                float* gates = sGates + (c & 3) * GATE_FLOATS;
+                const int r0 = lane, r1 = lane + 32;
+                float x = 0.f, y = 0.f, b0 = 0.f, b1 = 0.f;
+                if (r0 < R) { const size_t o = (size_t)(tok0 + c * C + r0) * H + h; x = __ldg(p.a + o); b0 = __ldg(p.beta + o); }
+                if (r1 < R) { const size_t o = (size_t)(tok0 + c * C + r1) * H + h; y = __ldg(p.a + o); b1 = __ldg(p.beta + o); }
+#pragma unroll
+                for (int d = 1; d < 32; d <<= 1) {
+                    const float xu = __shfl_up_sync(0xffffffffu, x, d);
+                    const float yu = __shfl_up_sync(0xffffffffu, y, d);
+                    if (lane >= d) { x += xu; y += yu; }
+                }
+                y += __shfl_sync(0xffffffffu, x, 31);
+                const float gC = __shfl_sync(0xffffffffu, y, 31);
+                if (c >= 4) wait(cta, B_GFREE0 + (c & 3), ((c >> 2) - 1) & 1);
+                gates[r0] = x * LOG2E; gates[r1] = y * LOG2E;                        // g_r log2(e)
+                gates[64 + r0] = b0; gates[64 + r1] = b1;                            // beta_r
+                gates[128 + r0] = ex2(x * LOG2E); gates[128 + r1] = ex2(y * LOG2E);  // e^{g_r}
+                gates[192 + r0] = ex2((gC - x) * LOG2E); gates[192 + r1] = ex2((gC - y) * LOG2E);
+                if (lane == 0) gates[256] = ex2(gC * LOG2E);
+                mbar_arrive(cta.bar(B_GREADY0 + (c & 3)));
             }
         } else if (warp == 13 && lane == 0) {
             // ---- TMA producer ----
