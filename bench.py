@@ -200,6 +200,12 @@ def run_ours(args):
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
 
     fn = gdn.gdn_chunk_prefill if cfg.dtype == "bf16" else gdn.gdn_chunk_prefill_f32
+    # scratch for the two-kernel pipeline (the library allocates nothing itself)
+    ws_bytes = 0
+    if cfg.dtype == "bf16" and not args.no_workspace:
+        ws_bytes = gdn.gdn_workspace_bytes(cfg.B, x.T_arg, cfg.H, cfg.d_k, cfg.d_v, cfg.packed)
+        if ws_bytes:
+            gdn.gdn_set_workspace(torch.empty(ws_bytes, dtype=torch.uint8, device=dev))
 
     def step():
         fn(d["q"], d["k"], d["v"], d["log_alpha"], d["beta"], d["initial_state"], out, fin, d["cu_seqlens"],
@@ -298,7 +304,8 @@ def run_ours(args):
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
                 "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True,
                 "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if cfg.dtype == "bf16" else "f32",
-                "data": "synthetic", "config": workload_config(cfg, x), "clocks": clocks, "e2e": e2e,
+                "data": "synthetic", "config": dict(workload_config(cfg, x), workspace_bytes=int(ws_bytes)),
+                "clocks": clocks, "e2e": e2e,
                 "gpu_launches": int(launches), "roofline": roofline, "cpu_baseline": cpu,
                 "ms_min": float(min(ms)), "ms_median": float(np.median(ms))}
         print(json.dumps(line), flush=True)
@@ -313,6 +320,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--workload", default="long", help="long (T=10240, the metric's configuration), short, serving, large")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-workspace", action="store_true", help="run the fused single-kernel path (no scratch)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

@@ -125,6 +125,22 @@ int gdn_chunk_prefill_host(const void* q_host, const void* k_host, const void* v
 size_t gdn_host_staging_bytes(int B, int T, int H, int d_k, int d_v);
 
 /*
+ * Optional scratch memory.  Without it gdn_chunk_prefill runs one fused kernel per call in
+ * which each (sequence, head) chain also does its own forward substitutions.  With scratch of
+ * at least gdn_workspace_bytes(...) bytes the state-independent steps (cumulative gate,
+ * token-token matrices, forward substitution, WY factor W) run first as a kernel over every
+ * (chunk, head) on all SMs -- "all C positions are solved together", Section "A chunked
+ * delta-rule scan for the recurrent layers" -- and leave their results in the scratch for the
+ * chain kernel; this is the faster path.  The scratch stays owned by the caller, is 256-byte
+ * aligned device memory, must outlive every call that uses it, and is shared by all calls
+ * (calls on different streams must not overlap).  gdn_set_workspace(NULL, 0) removes it.
+ * `packed` is 1 when cu_seqlens will be passed (T = total tokens), else 0.
+ * gdn_workspace_bytes returns 0 for sizes the tensor-core path does not support.
+ */
+size_t gdn_workspace_bytes(int B, int T, int H, int d_k, int d_v, int packed);
+int gdn_set_workspace(void* device_ptr, size_t bytes);
+
+/*
  * Waits for the device to finish (cudaDeviceSynchronize) and returns the status word of
  * the kernels: GDN_OK, or GDN_ERR_TIMEOUT if a bounded device-side wait (on a TMA copy,
  * a tensor-core completion or another warp role) ever expired, in which case the outputs

@@ -45,6 +45,12 @@ def lib():
         L.gdn_chunk_prefill_host.restype = i
         L.gdn_host_staging_bytes.argtypes = [i] * 5
         L.gdn_host_staging_bytes.restype = sz
+        L.gdn_workspace_bytes.argtypes = [i] * 6
+        L.gdn_workspace_bytes.restype = sz
+        L.gdn_set_workspace.argtypes = [vp, sz]
+        L.gdn_set_workspace.restype = i
+        L.gdn_debug_force_path.argtypes = [i]
+        L.gdn_debug_force_path.restype = None
         L.gdn_query_status.argtypes = []
         L.gdn_query_status.restype = i
         L.gdn_debug_set_dump.argtypes = [vp]
@@ -59,6 +65,29 @@ def lib():
 
 def gdn_status_string(status: int) -> str:
     return lib().gdn_status_string(int(status)).decode()
+
+
+def gdn_workspace_bytes(B: int, T: int, H: int, d_k: int, d_v: int, packed: bool = False) -> int:
+    return int(lib().gdn_workspace_bytes(B, T, H, d_k, d_v, 1 if packed else 0))
+
+
+_workspace_ref = None
+
+
+def gdn_set_workspace(workspace: Optional[torch.Tensor]) -> None:
+    """Hands the library a CUDA tensor to use as scratch (or None to remove it).  The binding
+    keeps a reference so the memory outlives the calls that use it."""
+    global _workspace_ref
+    if workspace is None:
+        rc = lib().gdn_set_workspace(None, 0)
+    else:
+        if workspace.device.type != "cuda" or not workspace.is_contiguous():
+            raise ValueError("workspace must be a contiguous CUDA tensor")
+        rc = lib().gdn_set_workspace(ctypes.c_void_p(workspace.data_ptr()),
+                                     workspace.numel() * workspace.element_size())
+    if rc != 0:
+        raise GdnError(rc, "gdn_set_workspace")
+    _workspace_ref = workspace
 
 
 def gdn_query_status() -> int:

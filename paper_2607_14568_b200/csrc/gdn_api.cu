@@ -31,9 +31,19 @@ PrefillArgs pack(const void* q, const void* k, const void* v, const float* log_a
     return PrefillArgs{q, k, v, log_alpha, beta, initial_state, out, final_state, cu_seqlens, B, T, H, d_k, d_v};
 }
 
+// Caller-provided scratch (gdn_set_workspace) and the path override used by the tests.
+void* g_workspace = nullptr;
+size_t g_workspace_bytes = 0;
+int g_force_path = 0;   // 0 = automatic, 1 = fused kernel, 2 = two-kernel pipeline
+
 int dispatch_bf16(const PrefillArgs& a, cudaStream_t stream) {
-    if (tc_supported(a.d_k, a.d_v)) return launch_tc(a, stream);
-    return launch_simt(a, /*io_bf16=*/true, stream);
+    if (!tc_supported(a.d_k, a.d_v)) return launch_simt(a, /*io_bf16=*/true, stream);
+    const uint64_t tokens = a.cu_seqlens ? (uint64_t)a.T : (uint64_t)a.B * a.T;
+    if (tokens == 0 || g_force_path == 1) return launch_tc(a, stream);
+    const size_t need = lean_workspace_bytes(a.B, a.T, a.H, a.d_k, a.d_v, a.cu_seqlens != nullptr);
+    if (g_workspace && g_workspace_bytes >= need) return launch_lean(a, g_workspace, g_workspace_bytes, stream);
+    if (g_force_path == 2) return GDN_ERR_WORKSPACE;
+    return launch_tc(a, stream);
 }
 
 inline size_t up256(size_t x) { return (x + 255) & ~(size_t)255; }
@@ -150,7 +160,21 @@ int gdn_chunk_prefill_host(const void* q_host, const void* k_host, const void* v
     return GDN_OK;
 }
 
+size_t gdn_workspace_bytes(int B, int T, int H, int d_k, int d_v, int packed) {
+    return lean_workspace_bytes(B, T, H, d_k, d_v, packed != 0);
+}
+
+int gdn_set_workspace(void* device_ptr, size_t bytes) {
+    if (device_ptr && (reinterpret_cast<uintptr_t>(device_ptr) & 255u)) return GDN_ERR_UNSUPPORTED;
+    g_workspace = device_ptr;
+    g_workspace_bytes = device_ptr ? bytes : 0;
+    return GDN_OK;
+}
+
 int gdn_query_status(void) { return tc_query_status(); }
+
+// Not part of the public header: 0 = automatic, 1 = fused kernel only, 2 = two-kernel pipeline only.
+void gdn_debug_force_path(int path) { g_force_path = path; }
 
 // Not part of the public header: lets the tests capture per-stage intermediates.
 void gdn_debug_set_dump(float* device_buffer) { tc_set_debug_dump(device_buffer); }

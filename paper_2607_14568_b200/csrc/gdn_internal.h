@@ -1,6 +1,7 @@
 // Internal declarations shared by the translation units of libgdn (not installed).
 #pragma once
 
+#include <cuda.h>
 #include <cuda_runtime.h>
 #include <cuda_bf16.h>
 #include <stdint.h>
@@ -34,6 +35,14 @@ int launch_tc(const PrefillArgs& a, cudaStream_t stream);
 bool tc_supported(int d_k, int d_v);
 int tc_query_status();               // synchronises the device, returns the kernels' status word
 void tc_set_debug_dump(float* p);    // tests only: stage dump of chunk 0 of CTA (0,0,0)
+
+// [tokens, H, d] bf16 tensor map, box = 64 tokens x 1 head x 64 features, 128-byte swizzle
+bool tc_make_map(CUtensorMap* map, const void* ptr, uint64_t tokens, uint64_t H, uint64_t d);
+
+// Two-kernel pipeline (prepare on all SMs, then the chain) using caller-provided scratch.
+size_t lean_workspace_bytes(int B, int T, int H, int d_k, int d_v, bool packed);
+int launch_lean(const PrefillArgs& a, void* workspace, size_t workspace_bytes, cudaStream_t stream);
+int lean_query_status();
 
 void count_launch(int n = 1);
 

@@ -1,0 +1,780 @@
+// Two-kernel tensor-core pipeline for bf16 storage (sm_100a), used when the caller has
+// provided scratch memory (gdn_set_workspace).
+//
+// The forward substitution is a latency-bound dependent chain; inside the fused kernel it
+// sits, once per chunk, on one warpgroup of the few SMs that own a (sequence, head) chain.
+// Here everything that does not depend on the incoming state is taken off those SMs:
+//
+//   gdn_prep_kernel    grid over every (chunk, head), all SMs, two CTAs per SM:
+//                      step a  cumulative log gate and the gate vectors,
+//                      step b1 G = [K;Q] K^T on the tensor core, decay masks -> A (fp32), P (bf16),
+//                      step b2 T = (I + A)^{-1}, blocked forward substitution in shared memory,
+//                      step b3 W^T = K^T (T diag(b e^g))^T on the tensor core,
+//                      and writes per (chunk, head) the operand images the chain needs:
+//                      -W^T, (T diag(b))^T, P (each already in the 128-byte-swizzled
+//                      shared-memory layout the MMA descriptors expect) and the gate vectors.
+//   gdn_chain_kernel   one CTA per (sequence, head, 128 value columns[, segment]): steps c and d.
+//                      TMA brings K, Q, V tiles and the images; U^T = V^T (T diag(b))^T,
+//                      v^T = U^T - S^T W^T, dS^T = (v e^{gC-g})^T K, O^T = e^g S^T Q^T + v^T P^T
+//                      run as tcgen05 MMAs with the state and v_new as TMEM A operands.
+//
+// (Section "A chunked delta-rule scan for the recurrent layers": state-independent work
+// for all positions at once, then a short recurrence over chunks.)
+//
+// Every wait is bounded (about a second); see gdn_tc.cu for the abort protocol.
+
+#include <cuda.h>
+
+#include "gdn_internal.h"
+#include "sm100_ptx.cuh"
+
+namespace gdn {
+
+__device__ int g_lean_status = 0;         // first non-zero status raised by these kernels
+
+namespace {
+
+using namespace ptx;
+
+constexpr int C = kChunk;
+constexpr int DK = 128;
+constexpr int DVB = 128;
+constexpr float LOG2E = 1.4426950408889634f;
+constexpr unsigned long long TIMEOUT_NS = 1000000000ull;
+
+// ---- per (chunk, head) scratch item ----
+constexpr uint32_t IT_W = 0;          // 16384: -W^T image   [d_k rows][64 r]
+constexpr uint32_t IT_T2 = 16384;     //  8192: (T diag(b))^T image [64 i][64 r]
+constexpr uint32_t IT_P = 24576;      //  8192: P image      [64 r][64 i]
+constexpr uint32_t IT_GATES = 32768;  //  1280: g log2e | beta | e^g | e^{gC-g} | e^{gC}
+constexpr uint32_t GATE_FLOATS = 320;
+constexpr uint32_t ITEM_BYTES = 34048;
+
+constexpr uint32_t LDA = 68, LDY = 36;
+
+struct Waiter {
+    uint32_t bars;              // shared address of barrier 0
+    volatile int* abort_flag;
+    __device__ __forceinline__ uint32_t bar(uint32_t i) const { return bars + i * 8; }
+    __device__ __forceinline__ void wait(uint32_t idx, uint32_t parity) const {
+        const uint32_t b = bar(idx);
+        if (mbar_try_wait(b, parity)) return;
+        const unsigned long long t0 = globaltimer_ns();
+        while (true) {
+            if (mbar_try_wait_suspend(b, parity, 100000u)) return;
+            if (*abort_flag) return;
+            if (globaltimer_ns() - t0 > TIMEOUT_NS) {
+                *abort_flag = 1;
+                atomicCAS(&g_lean_status, 0, (int)GDN_ERR_TIMEOUT);
+                return;
+            }
+        }
+    }
+};
+
+__device__ __forceinline__ uint32_t swz(uint32_t row, uint32_t chunk) {
+    return row * 128u + ((chunk ^ (row & 7u)) << 4);
+}
+__device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
+__device__ __forceinline__ void st_shared_f4(uint32_t addr, float a, float b, float c, float d) {
+    asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
+}
+__device__ __forceinline__ void st_global_v4(void* p, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+    *reinterpret_cast<uint4*>(p) = make_uint4(a, b, c, d);
+}
+// plain (untiled) bulk copy global -> shared; both addresses 16-byte aligned, size % 16 == 0
+__device__ __forceinline__ void bulk_load(uint32_t smem_dst, const void* gsrc, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(smem_dst), "l"(reinterpret_cast<uint64_t>(gsrc)), "r"(bytes), "r"(bar) : "memory");
+}
+
+// slot of chunk 0 of sequence n: disjoint ranges for any lengths, total <= tokens/64 + B
+__device__ __forceinline__ long slot_base(long tok0, int n) { return (tok0 >> 6) + n; }
+
+struct SeqInfo { long tok0; int len; };
+__device__ __forceinline__ SeqInfo seq_info(const int32_t* cu, int n, int T) {
+    SeqInfo s;
+    if (cu) { s.tok0 = cu[n]; s.len = cu[n + 1] - cu[n]; }
+    else    { s.tok0 = (long)n * T; s.len = T; }
+    return s;
+}
+
+// =====================================================================================
+// prepare kernel
+// =====================================================================================
+constexpr uint32_t PS_KQ = 0;                         // [K_lo | Q_lo | K_hi | Q_hi]
+constexpr uint32_t PS_T1 = 32768;                     // (T diag(b e^g))^T image
+constexpr uint32_t PS_A = PS_T1 + 8192;
+constexpr uint32_t PS_TF = PS_A + 64 * LDA * 4;
+constexpr uint32_t PS_Y = PS_TF + 64 * LDA * 4;
+constexpr uint32_t PS_GATES = PS_Y + 32 * LDY * 4;
+constexpr uint32_t PS_BARS = PS_GATES + GATE_FLOATS * 4;
+constexpr uint32_t PS_MISC = PS_BARS + 16 * 8;
+constexpr uint32_t PS_TOTAL = PS_MISC + 64;
+constexpr uint32_t PREP_SMEM = PS_TOTAL + 1024;
+constexpr int PREP_THREADS = 192;
+constexpr uint32_t PT_COLS = 64;
+
+enum PBar : uint32_t { PB_FULL = 0, PB_G, PB_W, PB_TREADY, PB_GREADY, PB_DONE };
+
+struct PrepParams {
+    const float* a;
+    const float* beta;
+    const int32_t* cu;
+    uint8_t* items;
+    long nslots;
+    int B, T, H;
+};
+
+constexpr uint32_t ID_G = make_idesc(128, 64, kFmtBF16, kFmtBF16, kMajorK, kMajorK);
+constexpr uint32_t ID_WU = make_idesc(128, 64, kFmtBF16, kFmtBF16, kMajorMN, kMajorMN);
+constexpr uint32_t ID_1 = make_idesc(128, 64, kFmtBF16, kFmtBF16, kMajorK, kMajorMN);
+constexpr uint32_t ID_O = make_idesc(128, 64, kFmtBF16, kFmtBF16, kMajorK, kMajorK);
+constexpr uint32_t ID_2 = make_idesc(128, 128, kFmtBF16, kFmtBF16, kMajorK, kMajorMN);
+
+__global__ void __launch_bounds__(PREP_THREADS, 2)
+gdn_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k, PrepParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* sm = smem_raw + (base - smem_u32(smem_raw));
+    float* sA = reinterpret_cast<float*>(sm + PS_A);
+    float* sTf = reinterpret_cast<float*>(sm + PS_TF);
+    float* sY = reinterpret_cast<float*>(sm + PS_Y);
+    float* gates = reinterpret_cast<float*>(sm + PS_GATES);
+    volatile uint32_t* sMisc = reinterpret_cast<volatile uint32_t*>(sm + PS_MISC);
+    Waiter w{base + PS_BARS, reinterpret_cast<volatile int*>(sm + PS_MISC + 4)};
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int H = p.H;
+    if (tid == 0) {
+        mbar_init(w.bar(PB_FULL), 1); mbar_init(w.bar(PB_G), 1); mbar_init(w.bar(PB_W), 1);
+        mbar_init(w.bar(PB_TREADY), 128); mbar_init(w.bar(PB_GREADY), 32); mbar_init(w.bar(PB_DONE), 128);
+        sMisc[1] = 0;
+        fence_mbar_init();
+    }
+    if (warp == 0) {
+        tmem_alloc(base + PS_MISC, PT_COLS);
+        tmem_relinquish();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem = sMisc[0];
+
+    const long nitems = p.nslots * H;
+    int it = 0;     // items this CTA has processed (barrier phases)
+    for (long item = blockIdx.x; item < nitems; item += gridDim.x) {
+        const long slot = item / H;
+        const int h = (int)(item - slot * H);
+        // which sequence owns this slot?  (largest n with slot_base(n) <= slot)
+        int n = 0;
+        if (p.cu) {
+            int lo = 0, hi = p.B - 1;
+            while (lo < hi) {
+                const int mid = (lo + hi + 1) >> 1;
+                if (slot_base(p.cu[mid], mid) <= slot) lo = mid; else hi = mid - 1;
+            }
+            n = lo;
+        } else {
+            int lo = 0, hi = p.B - 1;
+            while (lo < hi) {
+                const int mid = (lo + hi + 1) >> 1;
+                if (slot_base((long)mid * p.T, mid) <= slot) lo = mid; else hi = mid - 1;
+            }
+            n = lo;
+        }
+        const SeqInfo sq = seq_info(p.cu, n, p.T);
+        const int c = (int)(slot - slot_base(sq.tok0, n));
+        if (c * C >= sq.len) continue;                       // unused slot (uniform for the CTA)
+        const int R = min(C, sq.len - c * C);
+        const long tok = sq.tok0 + (long)c * C;
+        uint8_t* out_item = p.items + (size_t)item * ITEM_BYTES;
+        const uint32_t par = it & 1;
+
+        if (warp < 4) {
+            // ================= prepare warpgroup =================
+            const int tp = tid;
+            const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
+            w.wait(PB_GREADY, par);
+            w.wait(PB_G, par);
+            tc_fence_after_sync();
+            // ---- step b1: decay masks on G = [K;Q] K^T ----
+            {
+                const int r = tp & 63;
+                const float gr = gates[r];
+                const float br = gates[64 + r];
+                const bool is_a = tp < 64;
+                const int rmax = 32 * (warp & 1) + 31;
+                uint8_t* pimg = out_item + IT_P;
+#pragma unroll
+                for (int hh = 0; hh < 2; ++hh) {
+                    if (32 * hh <= rmax) {
+                        uint32_t x[32];
+                        tmem_ld32(tmem + lane_base + 32 * hh, x);
+                        tmem_wait_ld();
+                        float y[32];
+#pragma unroll
+                        for (int i4 = 0; i4 < 8; ++i4) {
+                            const float4 gi = *reinterpret_cast<const float4*>(gates + 32 * hh + 4 * i4);
+                            y[4 * i4 + 0] = ex2(gr - gi.x) * __uint_as_float(x[4 * i4 + 0]);
+                            y[4 * i4 + 1] = ex2(gr - gi.y) * __uint_as_float(x[4 * i4 + 1]);
+                            y[4 * i4 + 2] = ex2(gr - gi.z) * __uint_as_float(x[4 * i4 + 2]);
+                            y[4 * i4 + 3] = ex2(gr - gi.w) * __uint_as_float(x[4 * i4 + 3]);
+                        }
+                        if (is_a) {
+#pragma unroll
+                            for (int i4 = 0; i4 < 8; ++i4) {
+                                float o[4];
+#pragma unroll
+                                for (int e = 0; e < 4; ++e) {
+                                    const int i = 32 * hh + 4 * i4 + e;
+                                    o[e] = (i < r) ? br * y[4 * i4 + e] : 0.f;
+                                }
+                                st_shared_f4(base + PS_A + (r * LDA + 32 * hh + 4 * i4) * 4, o[0], o[1], o[2], o[3]);
+                            }
+                        } else {
+#pragma unroll
+                            for (int ch = 0; ch < 4; ++ch) {
+                                uint32_t pk[4];
+#pragma unroll
+                                for (int e = 0; e < 4; ++e) {
+                                    const int i0 = 32 * hh + 8 * ch + 2 * e;
+                                    pk[e] = pack_bf16((i0 <= r) ? y[8 * ch + 2 * e] : 0.f,
+                                                      (i0 + 1 <= r) ? y[8 * ch + 2 * e + 1] : 0.f);
+                                }
+                                st_global_v4(pimg + swz(r, 4 * hh + ch), pk[0], pk[1], pk[2], pk[3]);
+                            }
+                        }
+                    } else if (!is_a) {
+#pragma unroll
+                        for (int ch = 0; ch < 4; ++ch) st_global_v4(pimg + swz(r, 4 * hh + ch), 0u, 0u, 0u, 0u);
+                    }
+                }
+            }
+            named_bar_sync(1, 128);
+            // ---- step b2: T = (I + A)^{-1}, blocked forward substitution (fp32) ----
+            if (tp < 64) {   // level 0: four 16x16 diagonal blocks, one column per thread
+                const int I = tp >> 4, cc = tp & 15;
+                const float* Ab = sA + (16 * I) * LDA + 16 * I;
+                float* Tb = sTf + (16 * I) * LDA + 16 * I;
+                float xs[16];
+#pragma unroll
+                for (int r = 0; r < 16; ++r) {
+                    float acc0 = 0.f, acc1 = 0.f;
+#pragma unroll
+                    for (int i4 = 0; i4 < (r + 3) / 4; ++i4) {
+                        const float4 a4 = *reinterpret_cast<const float4*>(Ab + r * LDA + 4 * i4);
+                        if (4 * i4 + 0 < r) acc0 = fmaf(a4.x, xs[4 * i4 + 0], acc0);
+                        if (4 * i4 + 1 < r) acc1 = fmaf(a4.y, xs[4 * i4 + 1], acc1);
+                        if (4 * i4 + 2 < r) acc0 = fmaf(a4.z, xs[4 * i4 + 2], acc0);
+                        if (4 * i4 + 3 < r) acc1 = fmaf(a4.w, xs[4 * i4 + 3], acc1);
+                    }
+                    xs[r] = ((r == cc) ? 1.f : 0.f) - (acc0 + acc1);
+                    Tb[r * LDA + cc] = xs[r];
+                }
+            }
+            named_bar_sync(1, 128);
+            {   // level 1: 16-blocks (1,0) and (3,2):  T21 = -T22 (A21 T11)
+                const int pr = tp >> 6, r = (tp >> 2) & 15, cg = tp & 3;
+                const int lo = 32 * pr, hi = lo + 16;
+                float acc[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll 2
+                for (int i4 = 0; i4 < 4; ++i4) {
+                    const float4 a4 = *reinterpret_cast<const float4*>(sA + (hi + r) * LDA + lo + 4 * i4);
+                    const float av[4] = {a4.x, a4.y, a4.z, a4.w};
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const float4 t4 = *reinterpret_cast<const float4*>(sTf + (lo + 4 * i4 + e) * LDA + lo + 4 * cg);
+                        acc[0] = fmaf(av[e], t4.x, acc[0]); acc[1] = fmaf(av[e], t4.y, acc[1]);
+                        acc[2] = fmaf(av[e], t4.z, acc[2]); acc[3] = fmaf(av[e], t4.w, acc[3]);
+                    }
+                }
+                *reinterpret_cast<float4*>(sY + (16 * pr + r) * LDY + 4 * cg) = make_float4(acc[0], acc[1], acc[2], acc[3]);
+                named_bar_sync(1, 128);
+                float t[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll 2
+                for (int i4 = 0; i4 < 4; ++i4) {
+                    const float4 a4 = *reinterpret_cast<const float4*>(sTf + (hi + r) * LDA + hi + 4 * i4);
+                    const float av[4] = {a4.x, a4.y, a4.z, a4.w};
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const float4 y4 = *reinterpret_cast<const float4*>(sY + (16 * pr + 4 * i4 + e) * LDY + 4 * cg);
+                        t[0] = fmaf(av[e], y4.x, t[0]); t[1] = fmaf(av[e], y4.y, t[1]);
+                        t[2] = fmaf(av[e], y4.z, t[2]); t[3] = fmaf(av[e], y4.w, t[3]);
+                    }
+                }
+                *reinterpret_cast<float4*>(sTf + (hi + r) * LDA + lo + 4 * cg) = make_float4(-t[0], -t[1], -t[2], -t[3]);
+                *reinterpret_cast<float4*>(sTf + (lo + r) * LDA + hi + 4 * cg) = make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+            named_bar_sync(1, 128);
+            {   // level 2: the 32-block (1,0)
+                const int r = tp >> 2, cg = tp & 3;
+                float acc[8];
+#pragma unroll
+                for (int e = 0; e < 8; ++e) acc[e] = 0.f;
+#pragma unroll 2
+                for (int i4 = 0; i4 < 8; ++i4) {
+                    const float4 a4 = *reinterpret_cast<const float4*>(sA + (32 + r) * LDA + 4 * i4);
+                    const float av[4] = {a4.x, a4.y, a4.z, a4.w};
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const float* trow = sTf + (4 * i4 + e) * LDA + 8 * cg;
+                        const float4 t0 = *reinterpret_cast<const float4*>(trow);
+                        const float4 t1 = *reinterpret_cast<const float4*>(trow + 4);
+                        acc[0] = fmaf(av[e], t0.x, acc[0]); acc[1] = fmaf(av[e], t0.y, acc[1]);
+                        acc[2] = fmaf(av[e], t0.z, acc[2]); acc[3] = fmaf(av[e], t0.w, acc[3]);
+                        acc[4] = fmaf(av[e], t1.x, acc[4]); acc[5] = fmaf(av[e], t1.y, acc[5]);
+                        acc[6] = fmaf(av[e], t1.z, acc[6]); acc[7] = fmaf(av[e], t1.w, acc[7]);
+                    }
+                }
+                *reinterpret_cast<float4*>(sY + r * LDY + 8 * cg) = make_float4(acc[0], acc[1], acc[2], acc[3]);
+                *reinterpret_cast<float4*>(sY + r * LDY + 8 * cg + 4) = make_float4(acc[4], acc[5], acc[6], acc[7]);
+                named_bar_sync(1, 128);
+                float t[8];
+#pragma unroll
+                for (int e = 0; e < 8; ++e) t[e] = 0.f;
+#pragma unroll 2
+                for (int i4 = 0; i4 < 8; ++i4) {
+                    const float4 a4 = *reinterpret_cast<const float4*>(sTf + (32 + r) * LDA + 32 + 4 * i4);
+                    const float av[4] = {a4.x, a4.y, a4.z, a4.w};
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const float* yrow = sY + (4 * i4 + e) * LDY + 8 * cg;
+                        const float4 y0 = *reinterpret_cast<const float4*>(yrow);
+                        const float4 y1 = *reinterpret_cast<const float4*>(yrow + 4);
+                        t[0] = fmaf(av[e], y0.x, t[0]); t[1] = fmaf(av[e], y0.y, t[1]);
+                        t[2] = fmaf(av[e], y0.z, t[2]); t[3] = fmaf(av[e], y0.w, t[3]);
+                        t[4] = fmaf(av[e], y1.x, t[4]); t[5] = fmaf(av[e], y1.y, t[5]);
+                        t[6] = fmaf(av[e], y1.z, t[6]); t[7] = fmaf(av[e], y1.w, t[7]);
+                    }
+                }
+                *reinterpret_cast<float4*>(sTf + (32 + r) * LDA + 8 * cg) = make_float4(-t[0], -t[1], -t[2], -t[3]);
+                *reinterpret_cast<float4*>(sTf + (32 + r) * LDA + 8 * cg + 4) = make_float4(-t[4], -t[5], -t[6], -t[7]);
+            }
+            named_bar_sync(1, 128);
+            // ---- step b3 operands: row i = cc of (T diag(b e^g))^T (shared) and (T diag(b))^T (scratch) ----
+            {
+                const int cc = tp & 63, half = tp >> 6;
+                const float b = gates[64 + cc], bg = b * gates[128 + cc];
+                float t[32];
+#pragma unroll
+                for (int i = 0; i < 32; ++i)
+                    t[i] = (half == 0 && cc >= 32) ? 0.f : sTf[(32 * half + i) * LDA + cc];
+#pragma unroll
+                for (int ch = 0; ch < 4; ++ch) {
+                    uint32_t p1[4], p2[4];
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const float t0 = t[8 * ch + 2 * e], t1 = t[8 * ch + 2 * e + 1];
+                        p1[e] = pack_bf16(t0 * bg, t1 * bg);
+                        p2[e] = pack_bf16(t0 * b, t1 * b);
+                    }
+                    st_shared_v4(base + PS_T1 + swz(cc, 4 * half + ch), p1[0], p1[1], p1[2], p1[3]);
+                    st_global_v4(out_item + IT_T2 + swz(cc, 4 * half + ch), p2[0], p2[1], p2[2], p2[3]);
+                }
+            }
+            fence_proxy_async_smem();
+            tc_fence_before_sync();
+            mbar_arrive(w.bar(PB_TREADY));
+            // ---- step b3 result: -W^T image to scratch; gate vectors to scratch ----
+            if (tp < GATE_FLOATS / 4)
+                *reinterpret_cast<float4*>(out_item + IT_GATES + tp * 16) = *reinterpret_cast<const float4*>(gates + 4 * tp);
+            w.wait(PB_W, par);
+            tc_fence_after_sync();
+#pragma unroll
+            for (int hh = 0; hh < 2; ++hh) {
+                uint32_t x[32];
+                tmem_ld32(tmem + lane_base + 32 * hh, x);
+                tmem_wait_ld();
+#pragma unroll
+                for (int ch = 0; ch < 4; ++ch) {
+                    uint32_t pk[4];
+#pragma unroll
+                    for (int e = 0; e < 4; ++e)
+                        pk[e] = pack_bf16(-__uint_as_float(x[8 * ch + 2 * e]), -__uint_as_float(x[8 * ch + 2 * e + 1]));
+                    st_global_v4(out_item + IT_W + swz(tp, 4 * hh + ch), pk[0], pk[1], pk[2], pk[3]);
+                }
+            }
+            tc_fence_before_sync();
+            mbar_arrive(w.bar(PB_DONE));
+        } else if (warp == 4) {
+            // ================= TMA + MMA issue (one thread) =================
+            if (lane == 0) {
+                if (it > 0) w.wait(PB_DONE, (it - 1) & 1);          // shared memory and TMEM of the last item are free
+                tc_fence_after_sync();
+                const uint32_t kq = base + PS_KQ, full = w.bar(PB_FULL);
+                mbar_arrive_expect_tx(full, 32768);
+                tma_load_3d(kq, &map_k, 0, h, (int)tok, full);
+                tma_load_3d(kq + 8192, &map_q, 0, h, (int)tok, full);
+                tma_load_3d(kq + 16384, &map_k, 64, h, (int)tok, full);
+                tma_load_3d(kq + 24576, &map_q, 64, h, (int)tok, full);
+                w.wait(PB_FULL, par);
+#pragma unroll
+                for (uint32_t ks = 0; ks < 8; ++ks) {
+                    const uint32_t off = (ks >> 2) * 16384 + (ks & 3) * 32;
+                    mma_ss(tmem, make_smem_desc(kq + off, 16, 1024), make_smem_desc(kq + off, 16, 1024), ID_G, ks > 0);
+                }
+                mma_commit(w.bar(PB_G));
+                w.wait(PB_TREADY, par);
+                tc_fence_after_sync();
+#pragma unroll
+                for (uint32_t ks = 0; ks < 4; ++ks)
+                    mma_ss(tmem, make_smem_desc(kq + ks * 2048, 16384, 1024),
+                           make_smem_desc(base + PS_T1 + ks * 2048, 1024, 1024), ID_WU, ks > 0);
+                mma_commit(w.bar(PB_W));
+            }
+        } else {
+            // ================= step a: chunk-local cumulative log gate (one warp) =================
+            const int r0 = lane, r1 = lane + 32;
+            float x = 0.f, y = 0.f, b0 = 0.f, b1 = 0.f;
+            if (r0 < R) { const size_t o = (size_t)(tok + r0) * H + h; x = __ldg(p.a + o); b0 = __ldg(p.beta + o); }
+            if (r1 < R) { const size_t o = (size_t)(tok + r1) * H + h; y = __ldg(p.a + o); b1 = __ldg(p.beta + o); }
+#pragma unroll
+            for (int d = 1; d < 32; d <<= 1) {
+                const float xu = __shfl_up_sync(0xffffffffu, x, d);
+                const float yu = __shfl_up_sync(0xffffffffu, y, d);
+                if (lane >= d) { x += xu; y += yu; }
+            }
+            y += __shfl_sync(0xffffffffu, x, 31);
+            const float gC = __shfl_sync(0xffffffffu, y, 31);
+            if (it > 0) w.wait(PB_DONE, (it - 1) & 1);
+            gates[r0] = x * LOG2E; gates[r1] = y * LOG2E;
+            gates[64 + r0] = b0; gates[64 + r1] = b1;
+            gates[128 + r0] = ex2(x * LOG2E); gates[128 + r1] = ex2(y * LOG2E);
+            gates[192 + r0] = ex2((gC - x) * LOG2E); gates[192 + r1] = ex2((gC - y) * LOG2E);
+            gates[256 + lane] = (lane == 0) ? ex2(gC * LOG2E) : 0.f;
+            gates[288 + lane] = 0.f;
+            mbar_arrive(w.bar(PB_GREADY));
+        }
+        ++it;
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 0) {
+        tc_fence_after_sync();
+        tmem_dealloc(tmem, PT_COLS);
+    }
+}
+
+// =====================================================================================
+// chain kernel (steps c and d)
+// =====================================================================================
+constexpr int CHAIN_THREADS = 384;
+// tensor memory columns
+constexpr uint32_t TM_DV = 0, TM_DS = 64, TM_SBF = 192, TM_V = 256, TM_VT = 288, TM_O1 = 320, TM_O2 = 384;
+constexpr uint32_t CT_COLS = 512;
+// shared memory: two stages of {K/Q tiles, V tile, -W^T, T2, P, gates}
+constexpr uint32_t ST_KQ = 0, ST_V = 32768, ST_W = 49152, ST_T2 = 65536, ST_P = 73728, ST_GATES = 81920;
+constexpr uint32_t STAGE_BYTES = 83968;               // 82 KiB, multiple of 1024
+constexpr uint32_t STAGE_TX = 32768 + 16384 + 16384 + 8192 + 8192 + 1280;
+constexpr uint32_t CS_OST = 2 * STAGE_BYTES;           // bf16 output staging [64][128]
+constexpr uint32_t CS_BARS = CS_OST + 16384;
+constexpr uint32_t CS_MISC = CS_BARS + 16 * 8;
+constexpr uint32_t CS_TOTAL = CS_MISC + 64;
+constexpr uint32_t CHAIN_SMEM = CS_TOTAL + 1024;
+
+enum CBar : uint32_t { CB_FULL0 = 0, CB_FULL1, CB_FREE0, CB_FREE1, CB_V, CB_S, CB_O, CB_SREADY, CB_VREADY, CB_OFREE };
+
+struct ChainParams {
+    const float* s0;          // [N,H,d_k,d_v] or nullptr
+    __nv_bfloat16* out;
+    float* sT;
+    const int32_t* cu;
+    const uint8_t* items;
+    int B, T, H, dv;
+};
+
+__global__ void __launch_bounds__(CHAIN_THREADS, 1)
+gdn_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
+                 const __grid_constant__ CUtensorMap map_v, ChainParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* sm = smem_raw + (base - smem_u32(smem_raw));
+    volatile uint32_t* sMisc = reinterpret_cast<volatile uint32_t*>(sm + CS_MISC);
+    Waiter w{base + CS_BARS, reinterpret_cast<volatile int*>(sm + CS_MISC + 4)};
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int dvb = blockIdx.x, h = blockIdx.y, n = blockIdx.z;
+    const int H = p.H, dv = p.dv;
+    const SeqInfo sq = seq_info(p.cu, n, p.T);
+    const long tok0 = sq.tok0;
+    const int len = sq.len;
+    const int nchunks = (len + C - 1) / C;
+    const long slot0 = slot_base(tok0, n);
+
+    if (tid == 0) {
+        mbar_init(w.bar(CB_FULL0), 1); mbar_init(w.bar(CB_FULL1), 1);
+        mbar_init(w.bar(CB_FREE0), 257); mbar_init(w.bar(CB_FREE1), 257);   // MMA commit + chain + epilogue threads
+        mbar_init(w.bar(CB_V), 1); mbar_init(w.bar(CB_S), 1); mbar_init(w.bar(CB_O), 1);
+        mbar_init(w.bar(CB_SREADY), 128); mbar_init(w.bar(CB_VREADY), 128); mbar_init(w.bar(CB_OFREE), 128);
+        sMisc[1] = 0;
+        fence_mbar_init();
+    }
+    if (warp == 0) {
+        tmem_alloc(base + CS_MISC, CT_COLS);
+        tmem_relinquish();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem = sMisc[0];
+    const size_t state_off = ((size_t)n * H + h) * DK * dv + (size_t)dvb * DVB;
+
+    if (warp < 4) {
+        // =============================== chain warpgroup ===============================
+        setmaxnreg_inc<232>();
+        const int j = tid;
+        const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
+        float S[DK];
+        if (p.s0) {
+#pragma unroll
+            for (int m = 0; m < DK; ++m) S[m] = __ldg(p.s0 + state_off + (size_t)m * dv + j);
+        } else {
+#pragma unroll
+            for (int m = 0; m < DK; ++m) S[m] = 0.f;
+        }
+        if (nchunks > 0) {
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                uint32_t pk[16];
+#pragma unroll
+                for (int i = 0; i < 16; ++i) pk[i] = pack_bf16(S[32 * q + 2 * i], S[32 * q + 2 * i + 1]);
+                tmem_st16(tmem + lane_base + TM_SBF + 16 * q, pk);
+            }
+            tmem_wait_st();
+            tc_fence_before_sync();
+            mbar_arrive(w.bar(CB_SREADY));
+        }
+        for (int c = 0; c < nchunks; ++c) {
+            const uint32_t s = c & 1;
+            const float* gates = reinterpret_cast<const float*>(sm + s * STAGE_BYTES + ST_GATES);
+            w.wait(CB_V, c & 1);
+            tc_fence_after_sync();
+#pragma unroll
+            for (int hh = 0; hh < 2; ++hh) {
+                uint32_t x[32];
+                tmem_ld32(tmem + lane_base + TM_DV + 32 * hh, x);
+                tmem_wait_ld();
+                uint32_t pv[16], pd[16];
+#pragma unroll
+                for (int i = 0; i < 16; ++i) {
+                    const float v0 = __uint_as_float(x[2 * i]), v1 = __uint_as_float(x[2 * i + 1]);
+                    const float2 dec = *reinterpret_cast<const float2*>(gates + 192 + 32 * hh + 2 * i);
+                    pv[i] = pack_bf16(v0, v1);
+                    pd[i] = pack_bf16(v0 * dec.x, v1 * dec.y);
+                }
+                tmem_st16(tmem + lane_base + TM_V + 16 * hh, pv);
+                tmem_st16(tmem + lane_base + TM_VT + 16 * hh, pd);
+            }
+            tmem_wait_st();
+            tc_fence_before_sync();
+            mbar_arrive(w.bar(CB_VREADY));
+            w.wait(CB_S, c & 1);
+            tc_fence_after_sync();
+            const float gamma = gates[256];
+            mbar_arrive(w.bar(CB_FREE0 + s));          // last read of this stage by this thread
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                uint32_t d[32];
+                tmem_ld32(tmem + lane_base + TM_DS + 32 * q, d);
+                tmem_wait_ld();
+                uint32_t pk[16];
+#pragma unroll
+                for (int i = 0; i < 32; ++i) S[32 * q + i] = fmaf(gamma, S[32 * q + i], __uint_as_float(d[i]));
+#pragma unroll
+                for (int i = 0; i < 16; ++i) pk[i] = pack_bf16(S[32 * q + 2 * i], S[32 * q + 2 * i + 1]);
+                tmem_st16(tmem + lane_base + TM_SBF + 16 * q, pk);
+            }
+            tmem_wait_st();
+            tc_fence_before_sync();
+            mbar_arrive(w.bar(CB_SREADY));
+        }
+        if (p.sT) {
+#pragma unroll
+            for (int m = 0; m < DK; ++m) p.sT[state_off + (size_t)m * dv + j] = S[m];
+        }
+    } else if (warp < 8) {
+        // =============================== epilogue warpgroup ===============================
+        setmaxnreg_dec<96>();
+        const int j = tid - 128, we = j >> 5;
+        const uint32_t lane_base = (uint32_t)(we * 32) << 16;
+        __nv_bfloat16* ost = reinterpret_cast<__nv_bfloat16*>(sm + CS_OST);
+        for (int c = 0; c < nchunks; ++c) {
+            const uint32_t s = c & 1;
+            const int R = min(C, len - c * C);
+            const float* gates = reinterpret_cast<const float*>(sm + s * STAGE_BYTES + ST_GATES);
+            w.wait(CB_O, c & 1);
+            tc_fence_after_sync();
+#pragma unroll
+            for (int hh = 0; hh < 2; ++hh) {
+                uint32_t o1[32], o2[32];
+                tmem_ld32(tmem + lane_base + TM_O1 + 32 * hh, o1);
+                tmem_ld32(tmem + lane_base + TM_O2 + 32 * hh, o2);
+                tmem_wait_ld();
+                if (hh == 1) {
+                    tc_fence_before_sync();
+                    mbar_arrive(w.bar(CB_OFREE));
+                }
+#pragma unroll
+                for (int i = 0; i < 32; ++i) {
+                    const int r = 32 * hh + i;
+                    const float o = fmaf(gates[128 + r], __uint_as_float(o1[i]), __uint_as_float(o2[i]));
+                    ost[r * DVB + j] = __float2bfloat16_rn(o);
+                }
+            }
+            mbar_arrive(w.bar(CB_FREE0 + s));          // gate vectors of this stage no longer needed
+            named_bar_sync(2, 128);
+            {
+                __nv_bfloat16* obase = p.out + ((size_t)(tok0 + c * C) * H + h) * dv + (size_t)dvb * DVB;
+#pragma unroll
+                for (int it = 0; it < 8; ++it) {
+                    const int qd = it * 128 + j, r = qd >> 4, col = (qd & 15) * 8;
+                    if (r < R) {
+                        const uint4 val = *reinterpret_cast<const uint4*>(ost + r * DVB + col);
+                        *reinterpret_cast<uint4*>(obase + (size_t)r * H * dv + col) = val;
+                    }
+                }
+            }
+            named_bar_sync(2, 128);
+        }
+    } else {
+        // =============================== control warpgroup ===============================
+        setmaxnreg_dec<56>();
+        if (warp == 8 && lane == 0) {
+            // ---- MMA issuer ----
+            auto issue_U = [&](uint32_t s) {
+                const uint32_t vb = base + s * STAGE_BYTES + ST_V, t2 = base + s * STAGE_BYTES + ST_T2;
+#pragma unroll
+                for (uint32_t ks = 0; ks < 4; ++ks)
+                    mma_ss(tmem + TM_DV, make_smem_desc(vb + ks * 2048, 8192, 1024),
+                           make_smem_desc(t2 + ks * 2048, 1024, 1024), ID_WU, ks > 0);
+            };
+            if (nchunks > 0) {
+                w.wait(CB_FULL0, 0);
+                issue_U(0);
+            }
+            for (int c = 0; c < nchunks; ++c) {
+                const uint32_t s = c & 1, sb = base + s * STAGE_BYTES;
+                w.wait(CB_SREADY, c & 1);
+                tc_fence_after_sync();
+#pragma unroll
+                for (uint32_t ks = 0; ks < 8; ++ks)            // v^T = U^T - S^T W^T
+                    mma_ts(tmem + TM_DV, tmem + TM_SBF + ks * 8, make_smem_desc(sb + ST_W + ks * 2048, 1024, 1024), ID_1, 1);
+                mma_commit(w.bar(CB_V));
+                if (c > 0) { w.wait(CB_OFREE, (c - 1) & 1); tc_fence_after_sync(); }
+#pragma unroll
+                for (uint32_t ks = 0; ks < 8; ++ks)            // O1^T = S^T Q^T
+                    mma_ts(tmem + TM_O1, tmem + TM_SBF + ks * 8,
+                           make_smem_desc(sb + ST_KQ + 8192 + (ks >> 2) * 16384 + (ks & 3) * 32, 16, 1024), ID_O, ks > 0);
+                w.wait(CB_VREADY, c & 1);
+                tc_fence_after_sync();
+#pragma unroll
+                for (uint32_t ks = 0; ks < 4; ++ks)            // dS^T = (v e^{gC-g})^T K
+                    mma_ts(tmem + TM_DS, tmem + TM_VT + ks * 8, make_smem_desc(sb + ST_KQ + ks * 2048, 16384, 1024), ID_2, ks > 0);
+                mma_commit(w.bar(CB_S));
+#pragma unroll
+                for (uint32_t ks = 0; ks < 4; ++ks)            // O2^T = v^T P^T
+                    mma_ts(tmem + TM_O2, tmem + TM_V + ks * 8, make_smem_desc(sb + ST_P + ks * 32, 16, 1024), ID_O, ks > 0);
+                mma_commit(w.bar(CB_O));
+                mma_commit(w.bar(CB_FREE0 + s));
+                if (c + 1 < nchunks) {
+                    w.wait(CB_FULL0 + ((c + 1) & 1), ((c + 1) >> 1) & 1);
+                    issue_U((c + 1) & 1);                      // D_v is free: v_new of chunk c has been read
+                }
+            }
+        } else if (warp == 9 && lane == 0) {
+            // ---- TMA producer ----
+            prefetch_tensormap(&map_q);
+            prefetch_tensormap(&map_k);
+            prefetch_tensormap(&map_v);
+            for (int c = 0; c < nchunks; ++c) {
+                const uint32_t s = c & 1, sb = base + s * STAGE_BYTES;
+                if (c >= 2) w.wait(CB_FREE0 + s, ((c - 2) >> 1) & 1);
+                const uint32_t full = w.bar(CB_FULL0 + s);
+                const int tok = (int)(tok0 + (long)c * C);
+                const uint8_t* item = p.items + (size_t)((slot0 + c) * H + h) * ITEM_BYTES;
+                mbar_arrive_expect_tx(full, STAGE_TX);
+                tma_load_3d(sb + ST_KQ, &map_k, 0, h, tok, full);
+                tma_load_3d(sb + ST_KQ + 8192, &map_q, 0, h, tok, full);
+                tma_load_3d(sb + ST_KQ + 16384, &map_k, 64, h, tok, full);
+                tma_load_3d(sb + ST_KQ + 24576, &map_q, 64, h, tok, full);
+                tma_load_3d(sb + ST_V, &map_v, dvb * DVB, h, tok, full);
+                tma_load_3d(sb + ST_V + 8192, &map_v, dvb * DVB + 64, h, tok, full);
+                bulk_load(sb + ST_W, item + IT_W, 16384, full);
+                bulk_load(sb + ST_T2, item + IT_T2, 8192, full);
+                bulk_load(sb + ST_P, item + IT_P, 8192, full);
+                bulk_load(sb + ST_GATES, item + IT_GATES, 1280, full);
+            }
+            if (*w.abort_flag) {
+                for (int c = max(0, nchunks - 2); c < nchunks; ++c) {
+                    const uint32_t bar = w.bar(CB_FULL0 + (c & 1));
+                    const unsigned long long t0 = globaltimer_ns();
+                    while (!mbar_try_wait(bar, (c >> 1) & 1) && globaltimer_ns() - t0 < TIMEOUT_NS) {}
+                }
+            }
+        }
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 0) {
+        tc_fence_after_sync();
+        tmem_dealloc(tmem, CT_COLS);
+    }
+}
+
+}  // namespace
+
+// ------------------------------------------------------------------------------------------
+// host side
+// ------------------------------------------------------------------------------------------
+size_t lean_workspace_bytes(int B, int T, int H, int d_k, int d_v, bool packed) {
+    if (!tc_supported(d_k, d_v) || B <= 0 || T < 0 || H <= 0) return 0;
+    const size_t tokens = packed ? (size_t)T : (size_t)B * T;
+    const size_t slots = (tokens >> 6) + (size_t)B;
+    return slots * H * ITEM_BYTES;
+}
+
+int launch_lean(const PrefillArgs& a, void* workspace, size_t workspace_bytes, cudaStream_t stream) {
+    if (!tc_supported(a.d_k, a.d_v)) return GDN_ERR_UNSUPPORTED;
+    if (a.H > 65535 || a.B > 65535) return GDN_ERR_UNSUPPORTED;
+    const uint64_t tokens = a.cu_seqlens ? (uint64_t)a.T : (uint64_t)a.B * a.T;
+    const size_t need = lean_workspace_bytes(a.B, a.T, a.H, a.d_k, a.d_v, a.cu_seqlens != nullptr);
+    if (!workspace || workspace_bytes < need || (reinterpret_cast<uintptr_t>(workspace) & 255u)) return GDN_ERR_WORKSPACE;
+    CUtensorMap mq, mk, mv;
+    if (!tc_make_map(&mq, a.q, tokens, a.H, a.d_k) || !tc_make_map(&mk, a.k, tokens, a.H, a.d_k) ||
+        !tc_make_map(&mv, a.v, tokens, a.H, a.d_v))
+        return GDN_ERR_CUDA;
+    static int num_sms = 0;
+    if (num_sms == 0) {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+            return GDN_ERR_CUDA;
+    }
+    if (cudaFuncSetAttribute(gdn_prep_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)PREP_SMEM) != cudaSuccess ||
+        cudaFuncSetAttribute(gdn_chain_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)CHAIN_SMEM) != cudaSuccess)
+        return GDN_ERR_CUDA;
+    const long nslots = (long)(tokens >> 6) + a.B;
+    const long nitems = nslots * a.H;
+    PrepParams pp{a.log_alpha, a.beta, a.cu_seqlens, static_cast<uint8_t*>(workspace), nslots, a.B, a.T, a.H};
+    const int pgrid = (int)(nitems < 2L * num_sms ? nitems : 2L * num_sms);
+    gdn_prep_kernel<<<pgrid, PREP_THREADS, PREP_SMEM, stream>>>(mq, mk, pp);
+    count_launch();
+    if (cudaGetLastError() != cudaSuccess) return GDN_ERR_CUDA;
+    ChainParams cp{a.initial_state, static_cast<__nv_bfloat16*>(a.out), a.final_state, a.cu_seqlens,
+                   static_cast<const uint8_t*>(workspace), a.B, a.T, a.H, a.d_v};
+    dim3 grid(a.d_v / DVB, a.H, a.B);
+    gdn_chain_kernel<<<grid, CHAIN_THREADS, CHAIN_SMEM, stream>>>(mq, mk, mv, cp);
+    count_launch();
+    return cudaGetLastError() == cudaSuccess ? GDN_OK : GDN_ERR_CUDA;
+}
+
+int lean_query_status() {
+    int s = 0;
+    if (cudaMemcpyFromSymbol(&s, g_lean_status, sizeof(int)) != cudaSuccess) return GDN_ERR_CUDA;
+    return s;
+}
+
+}  // namespace gdn

@@ -762,6 +762,10 @@ bool make_map(CUtensorMap* map, const void* ptr, uint64_t tokens, uint64_t H, ui
 
 bool tc_supported(int d_k, int d_v) { return d_k == DK && d_v > 0 && d_v % DVB == 0; }
 
+bool tc_make_map(CUtensorMap* map, const void* ptr, uint64_t tokens, uint64_t H, uint64_t d) {
+    return make_map(map, ptr, tokens, H, d);
+}
+
 int launch_tc(const PrefillArgs& a, cudaStream_t stream) {
     if (!tc_supported(a.d_k, a.d_v)) return GDN_ERR_UNSUPPORTED;
     if (a.H > 65535 || a.B > 65535) return GDN_ERR_UNSUPPORTED;
@@ -796,7 +800,7 @@ int tc_query_status() {
     int s = 0;
     if (cudaDeviceSynchronize() != cudaSuccess) return GDN_ERR_CUDA;
     if (cudaMemcpyFromSymbol(&s, g_tc_status, sizeof(int)) != cudaSuccess) return GDN_ERR_CUDA;
-    return s;
+    return s ? s : lean_query_status();
 }
 
 void tc_set_debug_dump(float* p) { g_debug_dump = p; }

@@ -60,3 +60,35 @@ def assert_close(got, want, rel_tol, abs_tol=None, what=""):
     if abs_tol is not None:
         assert mx <= abs_tol, f"{what}: max-abs {mx:.3e} > {abs_tol:.1e} (rel-L2 {rel:.3e})"
     return rel, mx
+
+
+def _prefill_path(path):
+    """gdn_chunk_prefill pinned to one implementation: 1 = fused kernel, 2 = two-kernel pipeline
+    (with a freshly allocated workspace)."""
+    import paper_2607_14568_b200 as gdn
+
+    def fn(q, k, v, log_alpha, beta, initial_state, out, final_state, cu_seqlens=None, **kw):
+        if cu_seqlens is None:
+            B, T, H, d_k = q.shape
+        else:
+            T, H, d_k = q.shape
+            B = cu_seqlens.numel() - 1
+        ws = None
+        if path == 2:
+            nbytes = gdn.gdn_workspace_bytes(B, T, H, d_k, v.shape[-1], cu_seqlens is not None)
+            ws = torch.empty(max(nbytes, 256), dtype=torch.uint8, device=q.device)
+            gdn.gdn_set_workspace(ws)
+        gdn.lib().gdn_debug_force_path(path)
+        try:
+            r = gdn.gdn_chunk_prefill(q, k, v, log_alpha, beta, initial_state, out, final_state, cu_seqlens, **kw)
+            torch.cuda.synchronize()
+            assert gdn.gdn_query_status() == 0
+        finally:
+            gdn.lib().gdn_debug_force_path(0)
+            gdn.gdn_set_workspace(None)
+        return r
+    return fn
+
+
+prefill_fused = _prefill_path(1)
+prefill_two_kernel = _prefill_path(2)

@@ -8,12 +8,14 @@ import paper_2607_14568_b200 as gdn
 from workloads import chain_inputs, get_config, make_inputs, widen
 
 import oracle
-from gdn_testlib import (BF16_MAX_ABS, BF16_REL_L2, F32_REL_L2, assert_close, f64, run_lib, run_oracle,
-                         to_device)
+from gdn_testlib import (BF16_MAX_ABS, BF16_REL_L2, F32_REL_L2, assert_close, f64, prefill_fused,
+                         prefill_two_kernel, run_lib, run_oracle, to_device)
 
 pytestmark = pytest.mark.gpu
 
-BF16_FNS = {"main": gdn.gdn_chunk_prefill, "simt": gdn.gdn_chunk_prefill_bf16_simt}
+# "fused": one kernel per call (no scratch); "two_kernel": prepare kernel + chain kernel (scratch);
+# "simt": the fp32-arithmetic kernel with bf16 storage.
+BF16_FNS = {"fused": prefill_fused, "two_kernel": prefill_two_kernel, "simt": gdn.gdn_chunk_prefill_bf16_simt}
 
 
 def check_bf16(x, fn, what):
@@ -83,7 +85,7 @@ def test_f32_null_states_and_split_invariance():
 
 
 # ---- bf16 storage, reduced shapes that still span several tiles and a ragged tail ---------------
-@pytest.mark.parametrize("impl", ["main", "simt"])
+@pytest.mark.parametrize("impl", ["fused", "two_kernel", "simt"])
 @pytest.mark.parametrize("T,H,dv,init", [(64, 1, 128, 0.0), (200, 2, 128, 0.02), (1000, 2, 128, 0.02),
                                          (130, 2, 256, 0.0), (1, 1, 128, 0.02)])
 def test_bf16_reduced(impl, T, H, dv, init):
@@ -91,7 +93,7 @@ def test_bf16_reduced(impl, T, H, dv, init):
     check_bf16(make_inputs(cfg), BF16_FNS[impl], f"{impl} T={T}")
 
 
-@pytest.mark.parametrize("impl", ["main", "simt"])
+@pytest.mark.parametrize("impl", ["fused", "two_kernel", "simt"])
 def test_bf16_packed_ragged(impl):
     cfg = get_config("serving", B=5, H=2, lengths=(257, 64, 0, 1, 700), seed=31)
     x = make_inputs(cfg)
@@ -135,21 +137,23 @@ def test_deterministic():
 
 
 # ---- the benchmark configurations at full size ----------------------------------------------------
+@pytest.mark.parametrize("impl", ["fused", "two_kernel"])
 @pytest.mark.parametrize("name", ["short", "long", "serving"])
-def test_bf16_full_configs(name):
+def test_bf16_full_configs(name, impl):
     x = make_inputs(get_config(name))
-    (ro, mo), (rs, ms) = check_bf16(x, gdn.gdn_chunk_prefill, name)
-    print(f"\n{name}: out rel-L2 {ro:.2e} max-abs {mo:.2e}; state rel-L2 {rs:.2e} max-abs {ms:.2e}")
+    (ro, mo), (rs, ms) = check_bf16(x, BF16_FNS[impl], f"{name}/{impl}")
+    print(f"\n{name}/{impl}: out rel-L2 {ro:.2e} max-abs {mo:.2e}; state rel-L2 {rs:.2e} max-abs {ms:.2e}")
 
 
-def test_bf16_large_sampled_chains():
+@pytest.mark.parametrize("impl", ["fused", "two_kernel"])
+def test_bf16_large_sampled_chains(impl):
     """Configuration 'large' (B=4, T=32768, H=32, d_v=256) at full size; the oracle checks a seeded
     sample of whole (sequence, head) chains (heads are independent, so each checked chain is
     checked completely) and every other chain is checked for finiteness."""
     cfg = get_config("large")
     x = make_inputs(cfg, threads=16)
     d = to_device(x)
-    out, fin = run_lib(gdn.gdn_chunk_prefill, d)
+    out, fin = run_lib(BF16_FNS[impl], d)
     assert bool(torch.isfinite(out).all()) and bool(torch.isfinite(fin).all())
     rng = np.random.default_rng(5)
     chains = {(0, 0), (cfg.B - 1, cfg.H - 1)} | {(int(rng.integers(cfg.B)), int(rng.integers(cfg.H))) for _ in range(4)}
