@@ -51,6 +51,8 @@ def lib():
         L.gdn_set_workspace.restype = i
         L.gdn_debug_force_path.argtypes = [i]
         L.gdn_debug_force_path.restype = None
+        L.gdn_debug_force_segments.argtypes = [i]
+        L.gdn_debug_force_segments.restype = None
         L.gdn_query_status.argtypes = []
         L.gdn_query_status.restype = i
         L.gdn_debug_set_dump.argtypes = [vp]

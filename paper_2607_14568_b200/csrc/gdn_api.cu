@@ -176,6 +176,9 @@ int gdn_query_status(void) { return tc_query_status(); }
 // Not part of the public header: 0 = automatic, 1 = fused kernel only, 2 = two-kernel pipeline only.
 void gdn_debug_force_path(int path) { g_force_path = path; }
 
+// Not part of the public header: forces the number of sequence segments (0 = automatic).
+void gdn_debug_force_segments(int nseg) { lean_force_segments(nseg); }
+
 // Not part of the public header: lets the tests capture per-stage intermediates.
 void gdn_debug_set_dump(float* device_buffer) { tc_set_debug_dump(device_buffer); }
 

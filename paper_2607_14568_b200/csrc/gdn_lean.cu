@@ -31,6 +31,7 @@
 namespace gdn {
 
 __device__ int g_lean_status = 0;         // first non-zero status raised by these kernels
+static int g_lean_force_nseg = 0;         // tests: force a segment count (0 = automatic)
 
 namespace {
 
@@ -483,7 +484,9 @@ struct ChainParams {
     float* sT;
     const int32_t* cu;
     const uint8_t* items;
+    const float* seg_sin;     // [B*nseg, H, d_k, d_v] incoming states of segments 1.. (sequence split), or nullptr
     int B, T, H, dv;
+    int nseg, seg_chunks;     // segments per sequence (1 = no split) and chunks per segment
 };
 
 __global__ void __launch_bounds__(CHAIN_THREADS, 1)
@@ -496,13 +499,16 @@ gdn_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     Waiter w{base + CS_BARS, reinterpret_cast<volatile int*>(sm + CS_MISC + 4)};
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int dvb = blockIdx.x, h = blockIdx.y, n = blockIdx.z;
+    const int dvb = blockIdx.x, h = blockIdx.y;
+    const int n = blockIdx.z / p.nseg, seg = blockIdx.z % p.nseg;
     const int H = p.H, dv = p.dv;
     const SeqInfo sq = seq_info(p.cu, n, p.T);
-    const long tok0 = sq.tok0;
-    const int len = sq.len;
+    // this CTA walks chunks [seg * seg_chunks, ...) of the sequence
+    const int cbeg = seg * p.seg_chunks;
+    const long tok0 = sq.tok0 + (long)cbeg * C;
+    const int len = max(0, min(sq.len - cbeg * C, p.seg_chunks * C));
     const int nchunks = (len + C - 1) / C;
-    const long slot0 = slot_base(tok0, n);
+    const long slot0 = slot_base(sq.tok0, n) + cbeg;
 
     if (tid == 0) {
         mbar_init(w.bar(CB_FULL0), 1); mbar_init(w.bar(CB_FULL1), 1);
@@ -521,6 +527,8 @@ gdn_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     tc_fence_after_sync();
     const uint32_t tmem = sMisc[0];
     const size_t state_off = ((size_t)n * H + h) * DK * dv + (size_t)dvb * DVB;
+    const float* s_in = (seg == 0) ? (p.s0 ? p.s0 + state_off : nullptr)
+                                   : p.seg_sin + ((size_t)(n * p.nseg + seg) * H + h) * DK * dv + (size_t)dvb * DVB;
 
     if (warp < 4) {
         // =============================== chain warpgroup ===============================
@@ -528,9 +536,9 @@ gdn_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         const int j = tid;
         const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
         float S[DK];
-        if (p.s0) {
+        if (s_in) {
 #pragma unroll
-            for (int m = 0; m < DK; ++m) S[m] = __ldg(p.s0 + state_off + (size_t)m * dv + j);
+            for (int m = 0; m < DK; ++m) S[m] = __ldg(s_in + (size_t)m * dv + j);
         } else {
 #pragma unroll
             for (int m = 0; m < DK; ++m) S[m] = 0.f;
@@ -591,7 +599,7 @@ gdn_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             tc_fence_before_sync();
             mbar_arrive(w.bar(CB_SREADY));
         }
-        if (p.sT) {
+        if (p.sT && seg == p.nseg - 1) {
 #pragma unroll
             for (int m = 0; m < DK; ++m) p.sT[state_off + (size_t)m * dv + j] = S[m];
         }
@@ -724,23 +732,322 @@ gdn_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     }
 }
 
+
+// =====================================================================================
+// sequence split: segment summaries and their combination
+//
+// With few (sequence, head) chains the chain kernel leaves most SMs idle.  A sequence is
+// then cut into segments; every column s of the state obeys, over a segment,
+//     s_out = M_seg s_in + n_seg ,   M_seg = M_cL ... M_c1 ,  M_c = e^{gC} I - K~^T W
+// (the S^(c+1) = M_c S^(c) + N_c form of Section "A chunked delta-rule scan for the
+// recurrent layers", composed over the chunks of a segment).  gdn_summary_kernel runs,
+// per segment, the chain from a zero state (giving N_seg = n_seg for all value columns)
+// and the homogeneous chain from the identity (giving M_seg); gdn_combine_kernel walks
+// the segments in fp32, S_in[p+1] = M_p S_in[p] + N_p; the chain kernel then runs every
+// segment from its true incoming state.
+// =====================================================================================
+constexpr int SUM_THREADS = 384;
+constexpr uint32_t SS_K = 0, SS_V = 16384, SS_W = 32768, SS_T2 = 49152, SS_GATES = 57344;
+constexpr uint32_t SUM_STAGE = 59392;                       // 58 KiB
+constexpr uint32_t SUM_STAGE_TX = 16384 + 16384 + 16384 + 8192 + 1280;
+constexpr uint32_t SUM_STAGES = 3;
+constexpr uint32_t SUS_BARS = SUM_STAGES * SUM_STAGE;
+constexpr uint32_t SUS_MISC = SUS_BARS + 24 * 8;
+constexpr uint32_t SUM_SMEM = SUS_MISC + 64 + 1024;
+// tensor memory: instance 0 (values) and instance 1 (identity); bf16 state aliases the first
+// 64 columns of its own dS accumulator (read by MMA1 strictly before MMA2 overwrites it)
+__device__ __forceinline__ uint32_t sum_dv(int inst) { return inst ? 224u : 0u; }     // U^T / v_new^T
+__device__ __forceinline__ uint32_t sum_ds(int inst) { return inst ? 288u : 64u; }    // dS^T and bf16 S^T
+__device__ __forceinline__ uint32_t sum_vt(int inst) { return inst ? 416u : 192u; }   // bf16 decayed v_new^T
+constexpr uint32_t SUM_COLS = 512;
+
+enum SBar : uint32_t { SB_FULL0 = 0, SB_FREE0 = 3, SB_V0 = 6, SB_S0 = 8, SB_SREADY0 = 10, SB_VREADY0 = 12 };
+
+struct SummaryParams {
+    const int32_t* cu;
+    const uint8_t* items;
+    float* seg_n;             // [B*nseg, H, d_k, d_v]   N_seg
+    float* seg_mt;            // [B*nseg, H, d_k(i), d_k(m)]  M_seg transposed
+    int B, T, H, dv;
+    int nseg, seg_chunks;
+};
+
+__global__ void __launch_bounds__(SUM_THREADS, 1)
+gdn_summary_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
+                   SummaryParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* sm = smem_raw + (base - smem_u32(smem_raw));
+    volatile uint32_t* sMisc = reinterpret_cast<volatile uint32_t*>(sm + SUS_MISC);
+    Waiter w{base + SUS_BARS, reinterpret_cast<volatile int*>(sm + SUS_MISC + 4)};
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int dvb = blockIdx.x, h = blockIdx.y;
+    const int nsum = p.nseg - 1;                      // the last segment needs no summary
+    const int n = blockIdx.z / nsum, seg = blockIdx.z % nsum;
+    const int H = p.H, dv = p.dv;
+    const SeqInfo sq = seq_info(p.cu, n, p.T);
+    const int cbeg = seg * p.seg_chunks;
+    const long tok0 = sq.tok0 + (long)cbeg * C;
+    const int len = max(0, min(sq.len - cbeg * C, p.seg_chunks * C));
+    const int nchunks = (len + C - 1) / C;
+    const long slot0 = slot_base(sq.tok0, n) + cbeg;
+    const bool with_m = (dvb == 0);                   // M_seg does not depend on the value columns
+    const int ninst = with_m ? 2 : 1;
+
+    if (tid == 0) {
+        for (uint32_t i = 0; i < SUM_STAGES; ++i) {
+            mbar_init(w.bar(SB_FULL0 + i), 1);
+            mbar_init(w.bar(SB_FREE0 + i), 1 + 128 * ninst);
+        }
+        for (uint32_t i = 0; i < 2; ++i) {
+            mbar_init(w.bar(SB_V0 + i), 1); mbar_init(w.bar(SB_S0 + i), 1);
+            mbar_init(w.bar(SB_SREADY0 + i), 128); mbar_init(w.bar(SB_VREADY0 + i), 128);
+        }
+        sMisc[1] = 0;
+        fence_mbar_init();
+    }
+    if (warp == 0) {
+        tmem_alloc(base + SUS_MISC, SUM_COLS);
+        tmem_relinquish();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem = sMisc[0];
+
+    if (warp < 8) {
+        // ======================= two chain warpgroups: values (0) and identity (1) =======================
+        setmaxnreg_inc<224>();
+        const int inst = warp >> 2;
+        const int j = tid & 127;
+        const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
+        if (inst < ninst) {
+            float S[DK];
+#pragma unroll
+            for (int m = 0; m < DK; ++m) S[m] = (inst == 1 && m == j) ? 1.f : 0.f;
+            if (nchunks > 0) {
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    uint32_t pk[16];
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) pk[i] = pack_bf16(S[32 * q + 2 * i], S[32 * q + 2 * i + 1]);
+                    tmem_st16(tmem + lane_base + sum_ds(inst) + 16 * q, pk);
+                }
+                tmem_wait_st();
+                tc_fence_before_sync();
+                mbar_arrive(w.bar(SB_SREADY0 + inst));
+            }
+            for (int c = 0; c < nchunks; ++c) {
+                const uint32_t s = c % SUM_STAGES;
+                const float* gates = reinterpret_cast<const float*>(sm + s * SUM_STAGE + SS_GATES);
+                w.wait(SB_V0 + inst, c & 1);
+                tc_fence_after_sync();
+#pragma unroll
+                for (int hh = 0; hh < 2; ++hh) {
+                    uint32_t x[32];
+                    tmem_ld32(tmem + lane_base + sum_dv(inst) + 32 * hh, x);
+                    tmem_wait_ld();
+                    uint32_t pd[16];
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) {
+                        const float2 dec = *reinterpret_cast<const float2*>(gates + 192 + 32 * hh + 2 * i);
+                        pd[i] = pack_bf16(__uint_as_float(x[2 * i]) * dec.x, __uint_as_float(x[2 * i + 1]) * dec.y);
+                    }
+                    tmem_st16(tmem + lane_base + sum_vt(inst) + 16 * hh, pd);
+                }
+                tmem_wait_st();
+                tc_fence_before_sync();
+                mbar_arrive(w.bar(SB_VREADY0 + inst));
+                w.wait(SB_S0 + inst, c & 1);
+                tc_fence_after_sync();
+                const float gamma = gates[256];
+                mbar_arrive(w.bar(SB_FREE0 + s));
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    uint32_t d[32];
+                    tmem_ld32(tmem + lane_base + sum_ds(inst) + 32 * q, d);
+                    tmem_wait_ld();
+                    uint32_t pk[16];
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) S[32 * q + i] = fmaf(gamma, S[32 * q + i], __uint_as_float(d[i]));
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) pk[i] = pack_bf16(S[32 * q + 2 * i], S[32 * q + 2 * i + 1]);
+                    tmem_st16(tmem + lane_base + sum_ds(inst) + 16 * q, pk);   // columns already read
+                }
+                tmem_wait_st();
+                tc_fence_before_sync();
+                mbar_arrive(w.bar(SB_SREADY0 + inst));
+            }
+            const size_t sidx = (size_t)(n * p.nseg + seg) * H + h;
+            if (inst == 0) {
+                float* dst = p.seg_n + sidx * DK * dv + (size_t)dvb * DVB + j;       // [m][j]
+#pragma unroll
+                for (int m = 0; m < DK; ++m) dst[(size_t)m * dv] = S[m];
+            } else {
+                float4* dst = reinterpret_cast<float4*>(p.seg_mt + sidx * DK * DK + (size_t)j * DK);  // [i = j][m]
+#pragma unroll
+                for (int m4 = 0; m4 < DK / 4; ++m4) dst[m4] = make_float4(S[4 * m4], S[4 * m4 + 1], S[4 * m4 + 2], S[4 * m4 + 3]);
+            }
+        }
+    } else {
+        // =============================== control warpgroup ===============================
+        setmaxnreg_dec<56>();
+        if (warp == 8 && lane == 0) {
+            for (int c = 0; c < nchunks; ++c) {
+                const uint32_t s = c % SUM_STAGES, sb = base + s * SUM_STAGE;
+                w.wait(SB_FULL0 + s, (c / SUM_STAGES) & 1);
+                tc_fence_after_sync();
+#pragma unroll
+                for (uint32_t ks = 0; ks < 4; ++ks)            // U^T = V^T (T diag(b))^T
+                    mma_ss(tmem + sum_dv(0), make_smem_desc(sb + SS_V + ks * 2048, 8192, 1024),
+                           make_smem_desc(sb + SS_T2 + ks * 2048, 1024, 1024), ID_WU, ks > 0);
+                for (int inst = 0; inst < ninst; ++inst) {
+                    w.wait(SB_SREADY0 + inst, c & 1);
+                    tc_fence_after_sync();
+#pragma unroll
+                    for (uint32_t ks = 0; ks < 8; ++ks)        // v^T = U^T - S^T W^T   (U = 0 for the identity chain)
+                        mma_ts(tmem + sum_dv(inst), tmem + sum_ds(inst) + ks * 8,
+                               make_smem_desc(sb + SS_W + ks * 2048, 1024, 1024), ID_1, (inst == 0 || ks > 0) ? 1u : 0u);
+                    mma_commit(w.bar(SB_V0 + inst));
+                }
+                for (int inst = 0; inst < ninst; ++inst) {
+                    w.wait(SB_VREADY0 + inst, c & 1);
+                    tc_fence_after_sync();
+#pragma unroll
+                    for (uint32_t ks = 0; ks < 4; ++ks)        // dS^T = (v e^{gC-g})^T K
+                        mma_ts(tmem + sum_ds(inst), tmem + sum_vt(inst) + ks * 8,
+                               make_smem_desc(sb + SS_K + ks * 2048, 8192, 1024), ID_2, ks > 0);
+                    mma_commit(w.bar(SB_S0 + inst));
+                }
+                mma_commit(w.bar(SB_FREE0 + s));
+            }
+        } else if (warp == 9 && lane == 0) {
+            prefetch_tensormap(&map_k);
+            prefetch_tensormap(&map_v);
+            for (int c = 0; c < nchunks; ++c) {
+                const uint32_t s = c % SUM_STAGES, sb = base + s * SUM_STAGE;
+                if (c >= (int)SUM_STAGES) w.wait(SB_FREE0 + s, ((c / SUM_STAGES) - 1) & 1);
+                const uint32_t full = w.bar(SB_FULL0 + s);
+                const int tok = (int)(tok0 + (long)c * C);
+                const uint8_t* item = p.items + (size_t)((slot0 + c) * H + h) * ITEM_BYTES;
+                mbar_arrive_expect_tx(full, SUM_STAGE_TX);
+                tma_load_3d(sb + SS_K, &map_k, 0, h, tok, full);
+                tma_load_3d(sb + SS_K + 8192, &map_k, 64, h, tok, full);
+                tma_load_3d(sb + SS_V, &map_v, dvb * DVB, h, tok, full);
+                tma_load_3d(sb + SS_V + 8192, &map_v, dvb * DVB + 64, h, tok, full);
+                bulk_load(sb + SS_W, item + IT_W, 16384, full);
+                bulk_load(sb + SS_T2, item + IT_T2, 8192, full);
+                bulk_load(sb + SS_GATES, item + IT_GATES, 1280, full);
+            }
+            if (*w.abort_flag) {
+                for (int c = max(0, nchunks - (int)SUM_STAGES); c < nchunks; ++c) {
+                    const uint32_t bar = w.bar(SB_FULL0 + (c % SUM_STAGES));
+                    const unsigned long long t0 = globaltimer_ns();
+                    while (!mbar_try_wait(bar, (c / SUM_STAGES) & 1) && globaltimer_ns() - t0 < TIMEOUT_NS) {}
+                }
+            }
+        }
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 0) {
+        tc_fence_after_sync();
+        tmem_dealloc(tmem, SUM_COLS);
+    }
+}
+
+// S_in[p+1] = M_p S_in[p] + N_p in fp32, p = 0 .. nseg-2; one CTA per (sequence, head, 16 value columns).
+constexpr int CMB_COLS = 16;
+struct CombineParams {
+    const float* s0;          // [B, H, d_k, d_v] or nullptr
+    const float* seg_n;
+    const float* seg_mt;
+    float* seg_sin;
+    int H, dv, nseg;
+};
+
+__global__ void __launch_bounds__(256) gdn_combine_kernel(CombineParams p) {
+    __shared__ float sS[DK][CMB_COLS];
+    const int tid = threadIdx.x;
+    const int j0 = blockIdx.x * CMB_COLS, h = blockIdx.y, n = blockIdx.z;
+    const int H = p.H, dv = p.dv;
+    const int m = tid & 127, jh = tid >> 7;            // thread: state row m, 8 of the 16 columns
+    for (int idx = tid; idx < DK * CMB_COLS; idx += 256) {
+        const int i = idx / CMB_COLS, j = idx % CMB_COLS;
+        sS[i][j] = p.s0 ? p.s0[(((size_t)n * H + h) * DK + i) * dv + j0 + j] : 0.f;
+    }
+    __syncthreads();
+    for (int seg = 0; seg + 1 < p.nseg; ++seg) {
+        const size_t sidx = (size_t)(n * p.nseg + seg) * H + h;
+        const float* mt = p.seg_mt + sidx * DK * DK;              // [i][m]
+        const float* nn = p.seg_n + (sidx * DK + m) * dv + j0 + 8 * jh;
+        float acc[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) acc[e] = nn[e];
+#pragma unroll 8
+        for (int i = 0; i < DK; ++i) {
+            const float mv = __ldg(mt + (size_t)i * DK + m);
+            const float4 s0 = *reinterpret_cast<const float4*>(&sS[i][8 * jh]);
+            const float4 s1 = *reinterpret_cast<const float4*>(&sS[i][8 * jh + 4]);
+            acc[0] = fmaf(mv, s0.x, acc[0]); acc[1] = fmaf(mv, s0.y, acc[1]);
+            acc[2] = fmaf(mv, s0.z, acc[2]); acc[3] = fmaf(mv, s0.w, acc[3]);
+            acc[4] = fmaf(mv, s1.x, acc[4]); acc[5] = fmaf(mv, s1.y, acc[5]);
+            acc[6] = fmaf(mv, s1.z, acc[6]); acc[7] = fmaf(mv, s1.w, acc[7]);
+        }
+        __syncthreads();
+        float* dst = p.seg_sin + (((size_t)(n * p.nseg + seg + 1) * H + h) * DK + m) * dv + j0 + 8 * jh;
+#pragma unroll
+        for (int e = 0; e < 8; ++e) { sS[m][8 * jh + e] = acc[e]; dst[e] = acc[e]; }
+        __syncthreads();
+    }
+}
+
 }  // namespace
 
 // ------------------------------------------------------------------------------------------
 // host side
 // ------------------------------------------------------------------------------------------
+// Sequence split: only for batched (equal-length) input with few chains.  Returns the number
+// of segments per sequence (1 = no split) and the chunks per segment.
+static void plan_split(int B, int T, int H, int d_v, bool packed, int num_sms, int* nseg, int* seg_chunks) {
+    const int nch = (T + C - 1) / C;
+    *nseg = 1;
+    *seg_chunks = nch > 0 ? nch : 1;
+    if (packed || nch < 16) return;
+    const long chains = (long)B * H * (d_v / DVB);
+    if (chains * 2 > num_sms) return;
+    int want = (int)(num_sms / chains);
+    if (want > 16) want = 16;
+    if (want > nch / 4) want = nch / 4;                 // at least four chunks per segment
+    if (want < 2) return;
+    const int sc = (nch + want - 1) / want;
+    *seg_chunks = sc;
+    *nseg = (nch + sc - 1) / sc;
+}
+constexpr int kMaxSeg = 16;
+
 size_t lean_workspace_bytes(int B, int T, int H, int d_k, int d_v, bool packed) {
     if (!tc_supported(d_k, d_v) || B <= 0 || T < 0 || H <= 0) return 0;
     const size_t tokens = packed ? (size_t)T : (size_t)B * T;
     const size_t slots = (tokens >> 6) + (size_t)B;
-    return slots * H * ITEM_BYTES;
+    size_t bytes = slots * H * ITEM_BYTES;
+    bytes = (bytes + 255) & ~(size_t)255;
+    if (!packed) {
+        // split scratch, sized for the largest plan: incoming states, N_seg and M_seg^T per segment
+        const size_t per_seg = (size_t)B * H * d_k * (2 * (size_t)d_v + d_k) * sizeof(float);
+        const size_t chains = (size_t)B * H * (d_v / DVB);
+        if (chains * 2 <= 160) bytes += kMaxSeg * per_seg;
+    }
+    return bytes;
 }
 
 int launch_lean(const PrefillArgs& a, void* workspace, size_t workspace_bytes, cudaStream_t stream) {
     if (!tc_supported(a.d_k, a.d_v)) return GDN_ERR_UNSUPPORTED;
-    if (a.H > 65535 || a.B > 65535) return GDN_ERR_UNSUPPORTED;
-    const uint64_t tokens = a.cu_seqlens ? (uint64_t)a.T : (uint64_t)a.B * a.T;
-    const size_t need = lean_workspace_bytes(a.B, a.T, a.H, a.d_k, a.d_v, a.cu_seqlens != nullptr);
+    if (a.H > 65535 || a.B > 4095) return GDN_ERR_UNSUPPORTED;
+    const bool packed = a.cu_seqlens != nullptr;
+    const uint64_t tokens = packed ? (uint64_t)a.T : (uint64_t)a.B * a.T;
+    const size_t need = lean_workspace_bytes(a.B, a.T, a.H, a.d_k, a.d_v, packed);
     if (!workspace || workspace_bytes < need || (reinterpret_cast<uintptr_t>(workspace) & 255u)) return GDN_ERR_WORKSPACE;
     CUtensorMap mq, mk, mv;
     if (!tc_make_map(&mq, a.q, tokens, a.H, a.d_k) || !tc_make_map(&mk, a.k, tokens, a.H, a.d_k) ||
@@ -754,22 +1061,56 @@ int launch_lean(const PrefillArgs& a, void* workspace, size_t workspace_bytes, c
             return GDN_ERR_CUDA;
     }
     if (cudaFuncSetAttribute(gdn_prep_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)PREP_SMEM) != cudaSuccess ||
-        cudaFuncSetAttribute(gdn_chain_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)CHAIN_SMEM) != cudaSuccess)
+        cudaFuncSetAttribute(gdn_chain_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)CHAIN_SMEM) != cudaSuccess ||
+        cudaFuncSetAttribute(gdn_summary_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SUM_SMEM) != cudaSuccess)
         return GDN_ERR_CUDA;
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
     const long nslots = (long)(tokens >> 6) + a.B;
     const long nitems = nslots * a.H;
-    PrepParams pp{a.log_alpha, a.beta, a.cu_seqlens, static_cast<uint8_t*>(workspace), nslots, a.B, a.T, a.H};
+    // ---- state-independent steps, every (chunk, head) ----
+    PrepParams pp{a.log_alpha, a.beta, a.cu_seqlens, ws, nslots, a.B, a.T, a.H};
     const int pgrid = (int)(nitems < 2L * num_sms ? nitems : 2L * num_sms);
     gdn_prep_kernel<<<pgrid, PREP_THREADS, PREP_SMEM, stream>>>(mq, mk, pp);
     count_launch();
     if (cudaGetLastError() != cudaSuccess) return GDN_ERR_CUDA;
+    // ---- optional sequence split ----
+    int nseg = 1, seg_chunks = 1;
+    plan_split(a.B, a.T, a.H, a.d_v, packed, num_sms, &nseg, &seg_chunks);
+    if (g_lean_force_nseg > 0 && !packed) {           // tests: force a segment count
+        const int nch = (a.T + C - 1) / C;
+        nseg = g_lean_force_nseg > kMaxSeg ? kMaxSeg : g_lean_force_nseg;
+        if (nseg > nch) nseg = nch > 0 ? nch : 1;
+        seg_chunks = nch > 0 ? (nch + nseg - 1) / nseg : 1;
+        nseg = nch > 0 ? (nch + seg_chunks - 1) / seg_chunks : 1;
+    }
+    float* seg_sin = nullptr;
+    if (nseg > 1) {
+        const size_t items_bytes = ((size_t)nitems * ITEM_BYTES + 255) & ~(size_t)255;
+        const size_t state_elems = (size_t)a.B * nseg * a.H * a.d_k * a.d_v;
+        seg_sin = reinterpret_cast<float*>(ws + items_bytes);
+        float* seg_n = seg_sin + state_elems;
+        float* seg_mt = seg_n + state_elems;
+        SummaryParams sp{a.cu_seqlens, ws, seg_n, seg_mt, a.B, a.T, a.H, a.d_v, nseg, seg_chunks};
+        dim3 sgrid(a.d_v / DVB, a.H, a.B * (nseg - 1));
+        gdn_summary_kernel<<<sgrid, SUM_THREADS, SUM_SMEM, stream>>>(mk, mv, sp);
+        count_launch();
+        if (cudaGetLastError() != cudaSuccess) return GDN_ERR_CUDA;
+        CombineParams cb{a.initial_state, seg_n, seg_mt, seg_sin, a.H, a.d_v, nseg};
+        dim3 cgrid(a.d_v / CMB_COLS, a.H, a.B);
+        gdn_combine_kernel<<<cgrid, 256, 0, stream>>>(cb);
+        count_launch();
+        if (cudaGetLastError() != cudaSuccess) return GDN_ERR_CUDA;
+    }
+    // ---- steps c, d ----
     ChainParams cp{a.initial_state, static_cast<__nv_bfloat16*>(a.out), a.final_state, a.cu_seqlens,
-                   static_cast<const uint8_t*>(workspace), a.B, a.T, a.H, a.d_v};
-    dim3 grid(a.d_v / DVB, a.H, a.B);
+                   ws, seg_sin, a.B, a.T, a.H, a.d_v, nseg, seg_chunks};
+    dim3 grid(a.d_v / DVB, a.H, a.B * nseg);
     gdn_chain_kernel<<<grid, CHAIN_THREADS, CHAIN_SMEM, stream>>>(mq, mk, mv, cp);
     count_launch();
     return cudaGetLastError() == cudaSuccess ? GDN_OK : GDN_ERR_CUDA;
 }
+
+void lean_force_segments(int nseg) { g_lean_force_nseg = nseg; }
 
 int lean_query_status() {
     int s = 0;

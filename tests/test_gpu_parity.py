@@ -114,6 +114,21 @@ def test_bf16_packed_ragged(impl):
         assert torch.equal(o1[0], out[a:b]) and torch.equal(f1[0], fin[n])
 
 
+@pytest.mark.parametrize("T,nseg,gate", [(640, 2, 0.05), (1000, 3, 0.05), (2048, 5, 0.001), (4096, 16, 0.0),
+                                         (333, 4, 0.02)])
+def test_two_kernel_sequence_split(T, nseg, gate):
+    """The sequence split (segment summaries M, N; fp32 combination; per-segment chains) against the
+    oracle, including weak or no decay, where a segment's outgoing state depends fully on its
+    incoming one."""
+    cfg = get_config("long", T=T, H=2, gate_scale=gate, seed=60 + nseg)
+    x = make_inputs(cfg)
+    gdn.lib().gdn_debug_force_segments(nseg)
+    try:
+        check_bf16(x, prefill_two_kernel, f"split T={T} nseg={nseg}")
+    finally:
+        gdn.lib().gdn_debug_force_segments(0)
+
+
 def test_bf16_special_cases():
     """beta = 0 gives pure decay of the initial state; identity padding changes nothing."""
     cfg = get_config("long", T=192, H=2, seed=41)
