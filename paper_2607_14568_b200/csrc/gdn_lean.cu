@@ -957,8 +957,15 @@ gdn_summary_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
     }
 }
 
-// S_in[p+1] = M_p S_in[p] + N_p in fp32, p = 0 .. nseg-2; one CTA per (sequence, head, 16 value columns).
+// S_in[p+1] = M_p S_in[p] + N_p in fp32, p = 0 .. nseg-2; one CTA per (sequence, head, 16 value
+// columns).  M_p^T (64 KiB) is brought into shared memory by bulk copies, two segments ahead,
+// so the only serial cost per segment is the 128 x 128 x 16 product itself.
 constexpr int CMB_COLS = 16;
+constexpr int CMB_THREADS = 512;                       // 4 groups along the contraction x (32 x 4) tiles of 4 x 4
+constexpr uint32_t CMB_MT_BYTES = DK * DK * 4;
+constexpr uint32_t CMB_BUFS = 2;
+constexpr uint32_t CMB_S_BYTES = DK * CMB_COLS * 4;
+constexpr uint32_t CMB_SMEM = CMB_BUFS * CMB_MT_BYTES + 5 * CMB_S_BYTES + 64 + 128;
 struct CombineParams {
     const float* s0;          // [B, H, d_k, d_v] or nullptr
     const float* seg_n;
@@ -967,39 +974,84 @@ struct CombineParams {
     int H, dv, nseg;
 };
 
-__global__ void __launch_bounds__(256) gdn_combine_kernel(CombineParams p) {
-    __shared__ float sS[DK][CMB_COLS];
+__global__ void __launch_bounds__(CMB_THREADS) gdn_combine_kernel(CombineParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t base = (smem_u32(smem_raw) + 127u) & ~127u;
+    uint8_t* sm = smem_raw + (base - smem_u32(smem_raw));
+    const float* sMt = reinterpret_cast<const float*>(sm);                                   // [CMB_BUFS][i][m]
+    float (*sS)[CMB_COLS] = reinterpret_cast<float (*)[CMB_COLS]>(sm + CMB_BUFS * CMB_MT_BYTES);
+    float* sPart = reinterpret_cast<float*>(sm + CMB_BUFS * CMB_MT_BYTES + CMB_S_BYTES);     // [4][m][16]
+    const uint32_t misc = CMB_BUFS * CMB_MT_BYTES + 5 * CMB_S_BYTES;
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(sm + misc + 32);
+    Waiter w{base + misc, abort_flag};
+
     const int tid = threadIdx.x;
     const int j0 = blockIdx.x * CMB_COLS, h = blockIdx.y, n = blockIdx.z;
     const int H = p.H, dv = p.dv;
-    const int m = tid & 127, jh = tid >> 7;            // thread: state row m, 8 of the 16 columns
-    for (int idx = tid; idx < DK * CMB_COLS; idx += 256) {
+    const int kg = tid >> 7, mt4 = tid & 31, ct = (tid >> 5) & 3;     // product phase
+    const int rm = tid >> 2, rc = (tid & 3) * 4;                       // reduction phase: 4 outputs of row rm
+    auto load_mt = [&](int seg) {
+        const uint32_t buf = seg % CMB_BUFS, full = w.bar(buf);
+        const uint8_t* src = reinterpret_cast<const uint8_t*>(p.seg_mt + ((size_t)(n * p.nseg + seg) * H + h) * DK * DK);
+        mbar_arrive_expect_tx(full, CMB_MT_BYTES);
+#pragma unroll
+        for (uint32_t q = 0; q < 4; ++q)
+            bulk_load(base + buf * CMB_MT_BYTES + q * 16384, src + q * 16384, 16384, full);
+    };
+    if (tid == 0) {
+        for (uint32_t i = 0; i < CMB_BUFS; ++i) mbar_init(w.bar(i), 1);
+        *abort_flag = 0;
+        fence_mbar_init();
+    }
+    for (int idx = tid; idx < DK * CMB_COLS; idx += CMB_THREADS) {
         const int i = idx / CMB_COLS, j = idx % CMB_COLS;
         sS[i][j] = p.s0 ? p.s0[(((size_t)n * H + h) * DK + i) * dv + j0 + j] : 0.f;
     }
     __syncthreads();
+    if (tid == 0)
+        for (int sg = 0; sg < (int)CMB_BUFS && sg + 1 < p.nseg; ++sg) load_mt(sg);
+    auto n_ptr = [&](int seg) {
+        return p.seg_n + (((size_t)(n * p.nseg + seg) * H + h) * DK + rm) * dv + j0 + rc;
+    };
+    float4 nv = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (p.nseg > 1) nv = __ldg(reinterpret_cast<const float4*>(n_ptr(0)));
     for (int seg = 0; seg + 1 < p.nseg; ++seg) {
-        const size_t sidx = (size_t)(n * p.nseg + seg) * H + h;
-        const float* mt = p.seg_mt + sidx * DK * DK;              // [i][m]
-        const float* nn = p.seg_n + (sidx * DK + m) * dv + j0 + 8 * jh;
-        float acc[8];
+        const float4 ncur = nv;
+        if (seg + 2 < p.nseg) nv = __ldg(reinterpret_cast<const float4*>(n_ptr(seg + 1)));   // one hop ahead
+        w.wait(seg % CMB_BUFS, (seg / CMB_BUFS) & 1);
+        const float* mt = sMt + (seg % CMB_BUFS) * DK * DK + 4 * mt4;
+        float acc[4][4];
 #pragma unroll
-        for (int e = 0; e < 8; ++e) acc[e] = nn[e];
+        for (int r = 0; r < 4; ++r)
+#pragma unroll
+            for (int c = 0; c < 4; ++c) acc[r][c] = 0.f;
 #pragma unroll 8
-        for (int i = 0; i < DK; ++i) {
-            const float mv = __ldg(mt + (size_t)i * DK + m);
-            const float4 s0 = *reinterpret_cast<const float4*>(&sS[i][8 * jh]);
-            const float4 s1 = *reinterpret_cast<const float4*>(&sS[i][8 * jh + 4]);
-            acc[0] = fmaf(mv, s0.x, acc[0]); acc[1] = fmaf(mv, s0.y, acc[1]);
-            acc[2] = fmaf(mv, s0.z, acc[2]); acc[3] = fmaf(mv, s0.w, acc[3]);
-            acc[4] = fmaf(mv, s1.x, acc[4]); acc[5] = fmaf(mv, s1.y, acc[5]);
-            acc[6] = fmaf(mv, s1.z, acc[6]); acc[7] = fmaf(mv, s1.w, acc[7]);
-        }
-        __syncthreads();
-        float* dst = p.seg_sin + (((size_t)(n * p.nseg + seg + 1) * H + h) * DK + m) * dv + j0 + 8 * jh;
+        for (int ii = 0; ii < 32; ++ii) {
+            const int i = kg * 32 + ii;
+            const float4 a4 = *reinterpret_cast<const float4*>(mt + i * DK);
+            const float4 s4 = *reinterpret_cast<const float4*>(&sS[i][4 * ct]);
+            const float av[4] = {a4.x, a4.y, a4.z, a4.w}, sv[4] = {s4.x, s4.y, s4.z, s4.w};
 #pragma unroll
-        for (int e = 0; e < 8; ++e) { sS[m][8 * jh + e] = acc[e]; dst[e] = acc[e]; }
+            for (int r = 0; r < 4; ++r)
+#pragma unroll
+                for (int c = 0; c < 4; ++c) acc[r][c] = fmaf(av[r], sv[c], acc[r][c]);
+        }
+#pragma unroll
+        for (int r = 0; r < 4; ++r)
+            *reinterpret_cast<float4*>(sPart + (kg * DK + 4 * mt4 + r) * CMB_COLS + 4 * ct) =
+                make_float4(acc[r][0], acc[r][1], acc[r][2], acc[r][3]);
+        __syncthreads();                               // partial products done; sS and this M buffer are free
+        if (tid == 0 && seg + (int)CMB_BUFS < p.nseg - 1) load_mt(seg + CMB_BUFS);
+        float4 o = ncur;
+#pragma unroll
+        for (int g = 0; g < 4; ++g) {
+            const float4 q = *reinterpret_cast<const float4*>(sPart + (g * DK + rm) * CMB_COLS + rc);
+            o.x += q.x; o.y += q.y; o.z += q.z; o.w += q.w;
+        }
+        *reinterpret_cast<float4*>(&sS[rm][rc]) = o;
         __syncthreads();
+        // the global store drains while the next segment is being computed
+        *reinterpret_cast<float4*>(p.seg_sin + (((size_t)(n * p.nseg + seg + 1) * H + h) * DK + rm) * dv + j0 + rc) = o;
     }
 }
 
@@ -1062,7 +1114,8 @@ int launch_lean(const PrefillArgs& a, void* workspace, size_t workspace_bytes, c
     }
     if (cudaFuncSetAttribute(gdn_prep_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)PREP_SMEM) != cudaSuccess ||
         cudaFuncSetAttribute(gdn_chain_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)CHAIN_SMEM) != cudaSuccess ||
-        cudaFuncSetAttribute(gdn_summary_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SUM_SMEM) != cudaSuccess)
+        cudaFuncSetAttribute(gdn_summary_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SUM_SMEM) != cudaSuccess ||
+        cudaFuncSetAttribute(gdn_combine_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)CMB_SMEM) != cudaSuccess)
         return GDN_ERR_CUDA;
     uint8_t* ws = static_cast<uint8_t*>(workspace);
     const long nslots = (long)(tokens >> 6) + a.B;
@@ -1097,7 +1150,7 @@ int launch_lean(const PrefillArgs& a, void* workspace, size_t workspace_bytes, c
         if (cudaGetLastError() != cudaSuccess) return GDN_ERR_CUDA;
         CombineParams cb{a.initial_state, seg_n, seg_mt, seg_sin, a.H, a.d_v, nseg};
         dim3 cgrid(a.d_v / CMB_COLS, a.H, a.B);
-        gdn_combine_kernel<<<cgrid, 256, 0, stream>>>(cb);
+        gdn_combine_kernel<<<cgrid, CMB_THREADS, CMB_SMEM, stream>>>(cb);
         count_launch();
         if (cudaGetLastError() != cudaSuccess) return GDN_ERR_CUDA;
     }
