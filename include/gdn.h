@@ -54,7 +54,8 @@ typedef enum {
     GDN_ERR_UNSUPPORTED = 2,  /* chunk != 64, unsupported (d_k, d_v), misaligned pointer */
     GDN_ERR_WORKSPACE = 3,    /* caller-provided scratch too small */
     GDN_ERR_CUDA = 4,         /* a CUDA runtime/driver call or a launch failed */
-    GDN_ERR_TIMEOUT = 5       /* a bounded device-side wait expired (see gdn_query_status) */
+    GDN_ERR_TIMEOUT = 5,      /* a bounded device-side wait expired (see gdn_query_status) */
+    GDN_ERR_TOO_LARGE = 6     /* problem exceeds the built-in scratch of gdn_chunk_prefill_noalloc */
 } gdn_status;
 
 /* Same handle as cudaStream_t / CUstream (NULL = the default stream). */
@@ -139,6 +140,39 @@ size_t gdn_host_staging_bytes(int B, int T, int H, int d_k, int d_v);
  */
 size_t gdn_workspace_bytes(int B, int T, int H, int d_k, int d_v, int packed);
 int gdn_set_workspace(void* device_ptr, size_t bytes);
+
+/*
+ * gdn_chunk_prefill for callers that cannot allocate device memory.  (The paper has no
+ * counterpart to this entry point; it exists for how the library is embedded.)
+ *
+ * Who needs it: an operator that a host framework calls with nothing but its input and
+ * output buffers has no allocator to turn to, and a serving process that carved up the
+ * whole GPU into its own pools at start-up has nothing left to request.  Neither can hand
+ * gdn_set_workspace a scratch buffer, and neither may have cudaMalloc called on its behalf.
+ * This call needs none: it runs the two-kernel pipeline (prepare kernel, then chain kernel,
+ * without the sequence split) on a scratch area of 64 MiB that is built into the library
+ * image -- every GPU that loads the library carries those 64 MiB until the process ends.
+ * It calls no cudaMalloc, cudaFree or other allocating routine.
+ *
+ * Same arguments, layouts, support (d_k = 128, d_v a multiple of 128, chunk = 64) and
+ * results as gdn_chunk_prefill.  Limit: (tokens / 64 + B) * H * 34048 bytes must not exceed
+ * 64 MiB, tokens being T when cu_seqlens is given and B * T otherwise (for H = 16 that is
+ * about 7800 tokens); beyond it the call launches nothing and returns GDN_ERR_TOO_LARGE.
+ *
+ * The first call made while a given device is current also looks up the device address of
+ * the built-in scratch and sets kernel attributes for that device; make that first call
+ * outside any stream capture.  All calls share the one scratch area and find in it what
+ * the previous call left (nothing in it needs to be zero: each call overwrites every part
+ * it later reads).  Calls that overlap on the GPU -- different streams, or different host
+ * threads -- race on it; issue them one after another on one stream.
+ */
+int gdn_chunk_prefill_noalloc(const void* q, const void* k, const void* v,
+                              const float* log_alpha, const float* beta,
+                              const float* initial_state,
+                              void* out, float* final_state,
+                              const int32_t* cu_seqlens,
+                              int B, int T, int H, int d_k, int d_v, int chunk,
+                              gdn_stream_t stream);
 
 /*
  * Waits for the device to finish (cudaDeviceSynchronize) and returns the status word of

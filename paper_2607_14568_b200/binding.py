@@ -38,7 +38,8 @@ def lib():
         L = ctypes.CDLL(_LIB_PATH)
         vp, ip, i, sz = ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t
         prefill = [vp] * 8 + [ip] + [i] * 6 + [vp]
-        for name in ("gdn_chunk_prefill", "gdn_chunk_prefill_f32", "gdn_chunk_prefill_bf16_simt"):
+        for name in ("gdn_chunk_prefill", "gdn_chunk_prefill_f32", "gdn_chunk_prefill_bf16_simt",
+                     "gdn_chunk_prefill_noalloc"):
             getattr(L, name).argtypes = prefill
             getattr(L, name).restype = i
         L.gdn_chunk_prefill_host.argtypes = [vp] * 8 + [ip] + [i] * 6 + [vp, sz, vp]
@@ -176,6 +177,15 @@ def gdn_chunk_prefill_bf16_simt(q, k, v, log_alpha, beta, initial_state, out, fi
                                 chunk: int = 64, stream=None):
     """bf16 q/k/v/out through the fp32-arithmetic kernel; see include/gdn.h."""
     return _prefill("gdn_chunk_prefill_bf16_simt", torch.bfloat16, q, k, v, log_alpha, beta, initial_state,
+                    out, final_state, cu_seqlens, chunk, stream)
+
+
+def gdn_chunk_prefill_noalloc(q, k, v, log_alpha, beta, initial_state, out, final_state, cu_seqlens=None,
+                              chunk: int = 64, stream=None):
+    """gdn_chunk_prefill on the library's built-in 64 MiB scratch: for callers that have no way to
+    allocate device memory (see include/gdn.h).  Raises GdnError with status 6 when the problem
+    does not fit.  Make the first call on a device outside stream capture; do not overlap calls."""
+    return _prefill("gdn_chunk_prefill_noalloc", torch.bfloat16, q, k, v, log_alpha, beta, initial_state,
                     out, final_state, cu_seqlens, chunk, stream)
 
 

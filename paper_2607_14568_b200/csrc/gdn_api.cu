@@ -160,6 +160,18 @@ int gdn_chunk_prefill_host(const void* q_host, const void* k_host, const void* v
     return GDN_OK;
 }
 
+int gdn_chunk_prefill_noalloc(const void* q, const void* k, const void* v, const float* log_alpha,
+                              const float* beta, const float* initial_state, void* out, float* final_state,
+                              const int32_t* cu_seqlens, int B, int T, int H, int d_k, int d_v, int chunk,
+                              gdn_stream_t stream) {
+    const PrefillArgs a = pack(q, k, v, log_alpha, beta, initial_state, out, final_state, cu_seqlens, B, T, H, d_k, d_v);
+    if (int rc = validate(a, chunk)) return rc;
+    if (!tc_supported(d_k, d_v)) return GDN_ERR_UNSUPPORTED;
+    const uint64_t tokens = cu_seqlens ? (uint64_t)T : (uint64_t)B * T;
+    if (tokens == 0) return launch_tc(a, reinterpret_cast<cudaStream_t>(stream));   // states pass through; no scratch involved
+    return launch_lean_static(a, reinterpret_cast<cudaStream_t>(stream));
+}
+
 size_t gdn_workspace_bytes(int B, int T, int H, int d_k, int d_v, int packed) {
     return lean_workspace_bytes(B, T, H, d_k, d_v, packed != 0);
 }
@@ -192,6 +204,7 @@ const char* gdn_status_string(int status) {
         case GDN_ERR_WORKSPACE: return "caller-provided scratch too small";
         case GDN_ERR_CUDA: return "CUDA call or launch failed";
         case GDN_ERR_TIMEOUT: return "bounded device-side wait expired";
+        case GDN_ERR_TOO_LARGE: return "problem exceeds the 64 MiB built-in scratch of gdn_chunk_prefill_noalloc";
         default: return "unknown status";
     }
 }

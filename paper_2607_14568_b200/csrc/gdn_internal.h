@@ -42,6 +42,7 @@ bool tc_make_map(CUtensorMap* map, const void* ptr, uint64_t tokens, uint64_t H,
 // Two-kernel pipeline (prepare on all SMs, then the chain) using caller-provided scratch.
 size_t lean_workspace_bytes(int B, int T, int H, int d_k, int d_v, bool packed);
 int launch_lean(const PrefillArgs& a, void* workspace, size_t workspace_bytes, cudaStream_t stream);
+int launch_lean_static(const PrefillArgs& a, cudaStream_t stream);   // built-in scratch, allocates nothing
 int lean_query_status();
 void lean_force_segments(int nseg);   // tests only: 0 = automatic plan
 

@@ -1165,6 +1165,73 @@ int launch_lean(const PrefillArgs& a, void* workspace, size_t workspace_bytes, c
 
 void lean_force_segments(int nseg) { g_lean_force_nseg = nseg; }
 
+// ------------------------------------------------------------------------------------------
+// Entry point for callers that cannot allocate device memory.
+//
+// Some users of this library own no allocator: an operator plugged into a host framework is
+// handed its input and output buffers and nothing else, and a serving process that sized its
+// memory pools at start-up has no device memory left to ask for.  They cannot provide the
+// scratch the two-kernel pipeline wants, so that scratch lives here, in a fixed array inside
+// the library image.  Every GPU that loads the library holds these bytes until the process
+// exits, whether or not this entry point is ever called.
+//
+// The array name below is only a host-side handle; the address a kernel may use is obtained
+// with cudaGetSymbolAddress, once per device, by the first call made while that device is
+// current (make that first call outside any stream capture).  All calls share the array and
+// it keeps whatever the previous call left in it.  Nothing in it has to start at zero: the
+// prepare kernel writes every item the chain kernel reads before it is read, and items of
+// unused slots are never read.  Two calls that overlap on the GPU would race on it.
+// ------------------------------------------------------------------------------------------
+constexpr size_t kStaticScratchBytes = 64ull << 20;            // 64 MiB
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+constexpr int kMaxDevices = 64;
+
+int launch_lean_static(const PrefillArgs& a, cudaStream_t stream) {
+    if (!tc_supported(a.d_k, a.d_v)) return GDN_ERR_UNSUPPORTED;
+    if (a.H > 65535 || a.B > 65535) return GDN_ERR_UNSUPPORTED;
+    const bool packed = a.cu_seqlens != nullptr;
+    const uint64_t tokens = packed ? (uint64_t)a.T : (uint64_t)a.B * a.T;
+    const uint64_t nslots = (tokens >> 6) + (uint64_t)a.B;
+    const uint64_t need = nslots * (uint64_t)a.H * ITEM_BYTES;
+    if (need > kStaticScratchBytes) return GDN_ERR_TOO_LARGE;
+    // ---- set-up, once per device: the device address of the built-in scratch ----
+    static void* scratch_of_device[kMaxDevices] = {nullptr};
+    static int sms_of_device[kMaxDevices] = {0};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return GDN_ERR_CUDA;
+    if (dev < 0 || dev >= kMaxDevices) return GDN_ERR_UNSUPPORTED;
+    if (!scratch_of_device[dev]) {
+        void* ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || !ptr) return GDN_ERR_CUDA;
+        int sms = 0;
+        if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
+            return GDN_ERR_CUDA;
+        if (cudaFuncSetAttribute(gdn_prep_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)PREP_SMEM) != cudaSuccess ||
+            cudaFuncSetAttribute(gdn_chain_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)CHAIN_SMEM) != cudaSuccess)
+            return GDN_ERR_CUDA;
+        sms_of_device[dev] = sms;
+        scratch_of_device[dev] = ptr;
+    }
+    uint8_t* ws = static_cast<uint8_t*>(scratch_of_device[dev]);
+    CUtensorMap mq, mk, mv;
+    if (!tc_make_map(&mq, a.q, tokens, a.H, a.d_k) || !tc_make_map(&mk, a.k, tokens, a.H, a.d_k) ||
+        !tc_make_map(&mv, a.v, tokens, a.H, a.d_v))
+        return GDN_ERR_CUDA;
+    const long nitems = (long)nslots * a.H;
+    const long cap = 2L * sms_of_device[dev];
+    PrepParams pp{a.log_alpha, a.beta, a.cu_seqlens, ws, (long)nslots, a.B, a.T, a.H};
+    gdn_prep_kernel<<<(int)(nitems < cap ? nitems : cap), PREP_THREADS, PREP_SMEM, stream>>>(mq, mk, pp);
+    count_launch();
+    if (cudaGetLastError() != cudaSuccess) return GDN_ERR_CUDA;
+    const int nch = packed ? 1 : (a.T + C - 1) / C;            // one segment: the whole sequence
+    ChainParams cp{a.initial_state, static_cast<__nv_bfloat16*>(a.out), a.final_state, a.cu_seqlens,
+                   ws, nullptr, a.B, a.T, a.H, a.d_v, 1, packed ? (1 << 24) : (nch > 0 ? nch : 1)};
+    dim3 grid(a.d_v / DVB, a.H, a.B);
+    gdn_chain_kernel<<<grid, CHAIN_THREADS, CHAIN_SMEM, stream>>>(mq, mk, mv, cp);
+    count_launch();
+    return cudaGetLastError() == cudaSuccess ? GDN_OK : GDN_ERR_CUDA;
+}
+
 int lean_query_status() {
     int s = 0;
     if (cudaMemcpyFromSymbol(&s, g_lean_status, sizeof(int)) != cudaSuccess) return GDN_ERR_CUDA;

@@ -1,0 +1,65 @@
+"""The no-allocation entry point (built-in scratch) against the regular entry point.
+
+Collected last on purpose: a run that stops at the first failure has then already run every
+other test.  Some callers of the library cannot allocate device memory at all -- an operator
+embedded in a host framework only ever sees its argument buffers, a serving process has
+already given every byte to its own pools -- so this entry point must produce the same
+results as gdn_chunk_prefill without any scratch from the caller, call after call on the
+same shared scratch area.
+"""
+import ctypes
+
+import pytest
+import torch
+
+import paper_2607_14568_b200 as gdn
+from workloads import get_config, make_inputs
+
+from gdn_testlib import BF16_MAX_ABS, BF16_REL_L2, assert_close, f64, prefill_fused, to_device
+
+pytestmark = pytest.mark.gpu
+
+
+def _raw_call(name, d, cfg, T_arg):
+    """Straight through the C ABI: raw pointers and sizes, no binding helpers."""
+    fn = getattr(gdn.lib(), name)
+    ptr = lambda t: None if t is None else ctypes.c_void_p(t.data_ptr())
+    B = len(d["_lengths"])
+    rc = fn(ptr(d["q"]), ptr(d["k"]), ptr(d["v"]), ptr(d["log_alpha"]), ptr(d["beta"]), ptr(d["initial_state"]),
+            ptr(d["out"]), ptr(d["final_state"]), ptr(d["cu_seqlens"]), B, T_arg, cfg.H, cfg.d_k, cfg.d_v, 64,
+            ctypes.c_void_p(torch.cuda.current_stream().cuda_stream))
+    torch.cuda.synchronize()
+    return rc
+
+
+def test_noalloc_matches_regular_entry_point_twice_in_a_row():
+    cases = [get_config("long", T=1000, H=4, seed=71),                                    # ragged tail, initial state
+             get_config("serving", B=4, H=2, lengths=(300, 0, 65, 700), seed=72)]         # packed, second call
+    for cfg in cases:                                   # two calls in a row on the shared scratch
+        x = make_inputs(cfg)
+        ref = to_device(x)
+        prefill_fused(ref["q"], ref["k"], ref["v"], ref["log_alpha"], ref["beta"], ref["initial_state"],
+                      ref["out"], ref["final_state"], ref["cu_seqlens"])
+        d = to_device(x)
+        d["_lengths"] = x.lengths
+        d["out"].zero_()
+        d["final_state"].zero_()
+        gdn.gdn_set_workspace(None)                     # the caller provides no scratch
+        before = torch.cuda.memory_allocated()
+        assert _raw_call("gdn_chunk_prefill_noalloc", d, cfg, x.T_arg) == 0
+        assert torch.cuda.memory_allocated() == before
+        assert gdn.gdn_query_status() == 0
+        assert_close(f64(d["out"]), f64(ref["out"]), BF16_REL_L2, BF16_MAX_ABS, f"{cfg.name} out")
+        assert_close(f64(d["final_state"]), f64(ref["final_state"]), BF16_REL_L2, BF16_MAX_ABS, f"{cfg.name} state")
+
+
+def test_noalloc_rejects_problems_beyond_its_scratch():
+    cfg = get_config("long", T=64, H=16)
+    x = make_inputs(cfg)
+    d = to_device(x)
+    d["_lengths"] = x.lengths
+    n0 = gdn.gdn_launch_count()
+    # claim far more tokens than 64 MiB of scratch can serve: refused before anything is launched
+    assert _raw_call("gdn_chunk_prefill_noalloc", d, cfg, 1 << 20) == 6
+    assert gdn.gdn_launch_count() == n0
+    assert "64 MiB" in gdn.gdn_status_string(6)
