@@ -44,6 +44,37 @@ def algorithmic_work(cfg, lengths, with_initial_state):
             "bytes": tokens * H * bytes_per_th + state_bytes}
 
 
+def aggregate_over_ranks(local_ms, tokens_per_rank, steps, dist=None, device=None):
+    """Replicas-only aggregation: every rank ran `steps` steps over its own copy of the workload.
+    Job time = MAX over ranks of each local time; job tokens = sum over ranks.  `local_ms` is a
+    list of per-rank-local millisecond totals (e.g. [device-resident, end-to-end]); returns
+    (list of max-over-ranks ms, total tokens processed by the job)."""
+    import torch
+    world = dist.get_world_size() if dist is not None and dist.is_initialized() else 1
+    ms = [float(x) for x in local_ms]
+    tokens = float(tokens_per_rank) * steps
+    if world > 1:
+        t = torch.tensor(ms, dtype=torch.float64, device=device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = [float(x) for x in t]
+        n = torch.tensor([tokens], dtype=torch.float64, device=device)
+        dist.all_reduce(n, op=dist.ReduceOp.SUM)
+        tokens = float(n[0])
+    return ms, tokens
+
+
+def ncu_traffic_bytes(workload):
+    """DRAM bytes of one call (sum over its kernels) from the committed ncu summary, or None."""
+    path = os.path.join(ROOT, "profiles", f"{workload}_dram_traffic.txt")
+    if not os.path.exists(path):
+        return None
+    for line in open(path):
+        parts = line.split()
+        if len(parts) >= 2 and parts[0] == "total_bytes_per_call":
+            return float(parts[1])
+    return None
+
+
 def measured_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -268,16 +299,30 @@ def run_ours(args):
     else:
         e2e_ms, h2d, d2h = None, 0, 0
 
+    # ---- per-kernel breakdown (separate, untimed pass; events recorded inside the library) ----
+    kernels = None
+    if ws_bytes and gdn.lib().gdn_debug_set_timing(1) == 0:
+        import ctypes
+        acc = np.zeros(4)
+        buf = (ctypes.c_float * 4)()
+        for i in range(args.steps):
+            flush.fill_(i & 0xFF)
+            step()
+            if gdn.lib().gdn_debug_get_timing(buf) == 0:
+                acc += np.array(list(buf))
+        gdn.lib().gdn_debug_set_timing(0)
+        tot = float(acc.sum())
+        if tot > 0:
+            kernels = {n: {"ms": float(a) / args.steps, "share": float(a) / tot}
+                       for n, a in zip(("gdn_prep_kernel", "gdn_summary_kernel", "gdn_combine_kernel", "gdn_chain_kernel"), acc)}
+
     # ---- aggregate over ranks: max time, summed tokens ----
-    if world > 1:
-        t = torch.tensor([total_ms, e2e_ms or 0.0], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms, e2e_max = float(t[0]), float(t[1])
-        e2e_ms = e2e_max if e2e_ms is not None else None
-    tokens_all = work["tokens"] * world
-    value = tokens_all * args.steps / (total_ms * 1e-3)
+    (total_ms, e2e_max), tokens_job = aggregate_over_ranks([total_ms, e2e_ms or 0.0], work["tokens"], args.steps,
+                                                           dist if world > 1 else None, dev)
+    e2e_ms = e2e_max if e2e_ms is not None else None
+    value = tokens_job / (total_ms * 1e-3)
     if e2e_ms is not None:
-        e2e = {"value": tokens_all * args.steps / (e2e_ms * 1e-3), "unit": UNIT,
+        e2e = {"value": tokens_job / (e2e_ms * 1e-3), "unit": UNIT,
                "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h)}
 
     if rank == 0:
@@ -290,9 +335,11 @@ def run_ours(args):
             achieved, peak, unit = work["bytes"] / per_launch_s / 1e9, peaks["hbm_gbs"], "GB/s"
         else:
             achieved, peak, unit = work["flops"] / per_launch_s / 1e12, peaks["bf16_tflops"], "TFLOP/s"
+        dominant = max(kernels, key=lambda k: kernels[k]["ms"]) if kernels else None
         roofline = {"bound": bound, "achieved": achieved, "peak": peak, "unit": unit, "frac": achieved / peak,
-                    "traffic": None, "peak_source": peaks["source"],
-                    "kernel": "whole call (all kernels of one gdn_chunk_prefill)",
+                    "traffic": ncu_traffic_bytes(cfg.name), "peak_source": peaks["source"],
+                    "kernel": "whole call: algorithmic bytes of the path / time of all kernels of one gdn_chunk_prefill",
+                    "kernels": kernels, "dominant_kernel": dominant,
                     "algorithmic_bytes": work["bytes"], "algorithmic_flops": work["flops"],
                     "roofline_us": 1e6 * max(t_hbm, t_tc)}
         # CPU baseline: the oracle as it stands, bounded sample, host cores

@@ -52,6 +52,10 @@ def lib():
         L.gdn_set_workspace.restype = i
         L.gdn_debug_force_path.argtypes = [i]
         L.gdn_debug_force_path.restype = None
+        L.gdn_debug_set_timing.argtypes = [i]
+        L.gdn_debug_set_timing.restype = i
+        L.gdn_debug_get_timing.argtypes = [ctypes.POINTER(ctypes.c_float)]
+        L.gdn_debug_get_timing.restype = i
         L.gdn_debug_force_segments.argtypes = [i]
         L.gdn_debug_force_segments.restype = None
         L.gdn_query_status.argtypes = []

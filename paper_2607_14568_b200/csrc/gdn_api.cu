@@ -188,6 +188,10 @@ int gdn_query_status(void) { return tc_query_status(); }
 // Not part of the public header: 0 = automatic, 1 = fused kernel only, 2 = two-kernel pipeline only.
 void gdn_debug_force_path(int path) { g_force_path = path; }
 
+// Not part of the public header: per-kernel event timing of the two-kernel pipeline (benchmark).
+int gdn_debug_set_timing(int enable) { return lean_set_timing(enable); }
+int gdn_debug_get_timing(float* ms4) { return ms4 ? lean_get_timing(ms4) : GDN_ERR_INVALID_ARG; }
+
 // Not part of the public header: forces the number of sequence segments (0 = automatic).
 void gdn_debug_force_segments(int nseg) { lean_force_segments(nseg); }
 

@@ -32,6 +32,11 @@ namespace gdn {
 
 __device__ int g_lean_status = 0;         // first non-zero status raised by these kernels
 static int g_lean_force_nseg = 0;         // tests: force a segment count (0 = automatic)
+// optional per-kernel timing of the two-kernel pipeline (benchmark only): five events around the
+// prepare, summary, combine and chain kernels of the most recent call
+static bool g_lean_timing = false;
+static cudaEvent_t g_lean_events[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};
+static bool g_lean_split_last = false;
 
 namespace {
 
@@ -1123,9 +1128,12 @@ int launch_lean(const PrefillArgs& a, void* workspace, size_t workspace_bytes, c
     // ---- state-independent steps, every (chunk, head) ----
     PrepParams pp{a.log_alpha, a.beta, a.cu_seqlens, ws, nslots, a.B, a.T, a.H};
     const int pgrid = (int)(nitems < 2L * num_sms ? nitems : 2L * num_sms);
+    auto mark = [&](int i) { if (g_lean_timing && g_lean_events[i]) cudaEventRecord(g_lean_events[i], stream); };
+    mark(0);
     gdn_prep_kernel<<<pgrid, PREP_THREADS, PREP_SMEM, stream>>>(mq, mk, pp);
     count_launch();
     if (cudaGetLastError() != cudaSuccess) return GDN_ERR_CUDA;
+    mark(1);
     // ---- optional sequence split ----
     int nseg = 1, seg_chunks = 1;
     plan_split(a.B, a.T, a.H, a.d_v, packed, num_sms, &nseg, &seg_chunks);
@@ -1148,22 +1156,50 @@ int launch_lean(const PrefillArgs& a, void* workspace, size_t workspace_bytes, c
         gdn_summary_kernel<<<sgrid, SUM_THREADS, SUM_SMEM, stream>>>(mk, mv, sp);
         count_launch();
         if (cudaGetLastError() != cudaSuccess) return GDN_ERR_CUDA;
+        mark(2);
         CombineParams cb{a.initial_state, seg_n, seg_mt, seg_sin, a.H, a.d_v, nseg};
         dim3 cgrid(a.d_v / CMB_COLS, a.H, a.B);
         gdn_combine_kernel<<<cgrid, CMB_THREADS, CMB_SMEM, stream>>>(cb);
         count_launch();
         if (cudaGetLastError() != cudaSuccess) return GDN_ERR_CUDA;
+        mark(3);
     }
+    g_lean_split_last = nseg > 1;
     // ---- steps c, d ----
     ChainParams cp{a.initial_state, static_cast<__nv_bfloat16*>(a.out), a.final_state, a.cu_seqlens,
                    ws, seg_sin, a.B, a.T, a.H, a.d_v, nseg, seg_chunks};
     dim3 grid(a.d_v / DVB, a.H, a.B * nseg);
     gdn_chain_kernel<<<grid, CHAIN_THREADS, CHAIN_SMEM, stream>>>(mq, mk, mv, cp);
     count_launch();
+    mark(4);
     return cudaGetLastError() == cudaSuccess ? GDN_OK : GDN_ERR_CUDA;
 }
 
 void lean_force_segments(int nseg) { g_lean_force_nseg = nseg; }
+
+int lean_set_timing(int enable) {
+    if (enable)
+        for (auto& e : g_lean_events)
+            if (!e && cudaEventCreate(&e) != cudaSuccess) return GDN_ERR_CUDA;
+    g_lean_timing = enable != 0;
+    return GDN_OK;
+}
+
+// milliseconds of {prepare, summary, combine, chain} of the most recent call (0 for kernels not run)
+int lean_get_timing(float* ms4) {
+    for (int i = 0; i < 4; ++i) ms4[i] = 0.f;
+    if (!g_lean_events[0]) return GDN_ERR_INVALID_ARG;
+    if (cudaEventSynchronize(g_lean_events[4]) != cudaSuccess) return GDN_ERR_CUDA;
+    bool ok = cudaEventElapsedTime(&ms4[0], g_lean_events[0], g_lean_events[1]) == cudaSuccess;
+    if (g_lean_split_last) {
+        ok = ok && cudaEventElapsedTime(&ms4[1], g_lean_events[1], g_lean_events[2]) == cudaSuccess;
+        ok = ok && cudaEventElapsedTime(&ms4[2], g_lean_events[2], g_lean_events[3]) == cudaSuccess;
+        ok = ok && cudaEventElapsedTime(&ms4[3], g_lean_events[3], g_lean_events[4]) == cudaSuccess;
+    } else {
+        ok = ok && cudaEventElapsedTime(&ms4[3], g_lean_events[1], g_lean_events[4]) == cudaSuccess;
+    }
+    return ok ? GDN_OK : GDN_ERR_CUDA;
+}
 
 // ------------------------------------------------------------------------------------------
 // Entry point for callers that cannot allocate device memory.
