@@ -197,6 +197,7 @@ void gdn_debug_force_segments(int nseg) { lean_force_segments(nseg); }
 
 // Not part of the public header: lets the tests capture per-stage intermediates.
 void gdn_debug_set_dump(float* device_buffer) { tc_set_debug_dump(device_buffer); }
+void gdn_debug_set_chain_stamps(float* device_buffer) { lean_set_debug(device_buffer); }
 
 unsigned long long gdn_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 

@@ -37,6 +37,7 @@ static int g_lean_force_nseg = 0;         // tests: force a segment count (0 = a
 static bool g_lean_timing = false;
 static cudaEvent_t g_lean_events[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};
 static bool g_lean_split_last = false;
+static float* g_lean_dbg = nullptr;        // debug: time stamps of the chain kernel
 
 namespace {
 
@@ -62,6 +63,15 @@ struct Waiter {
     uint32_t bars;              // shared address of barrier 0
     volatile int* abort_flag;
     __device__ __forceinline__ uint32_t bar(uint32_t i) const { return bars + i * 8; }
+    // For waits on the sequential chain: poll without suspending for a short while (a suspended
+    // thread wakes up late), then fall back to the bounded suspending wait.
+    __device__ __forceinline__ void wait_hot(uint32_t idx, uint32_t parity) const {
+        const uint32_t b = bar(idx);
+#pragma unroll 1
+        for (int i = 0; i < 4096; ++i)
+            if (mbar_try_wait(b, parity)) return;
+        wait(idx, parity);
+    }
     __device__ __forceinline__ void wait(uint32_t idx, uint32_t parity) const {
         const uint32_t b = bar(idx);
         if (mbar_try_wait(b, parity)) return;
@@ -472,16 +482,25 @@ constexpr int CHAIN_THREADS = 384;
 constexpr uint32_t TM_DV = 0, TM_DS = 64, TM_SBF = 192, TM_V = 256, TM_VT = 288, TM_O1 = 320, TM_O2 = 384;
 constexpr uint32_t CT_COLS = 512;
 // shared memory: two stages of {K/Q tiles, V tile, -W^T, T2, P, gates}
-constexpr uint32_t ST_KQ = 0, ST_V = 32768, ST_W = 49152, ST_T2 = 65536, ST_P = 73728, ST_GATES = 81920;
-constexpr uint32_t STAGE_BYTES = 83968;               // 82 KiB, multiple of 1024
-constexpr uint32_t STAGE_TX = 32768 + 16384 + 16384 + 8192 + 8192 + 1280;
-constexpr uint32_t CS_OST = 2 * STAGE_BYTES;           // bf16 output staging [64][128]
+// shared memory: operands are staged in two rings with different lifetimes.
+//   ring A (2 deep): K/Q tiles, -W^T, P   -- used from the v_new MMA of a chunk to its last output MMA
+//   ring B (3 deep): V tile, (T diag b)^T -- used only by the U^T MMA, which is issued one chunk early
+//   gate vectors (4 deep): read by threads, not by MMAs; a slot is reused four chunks later, when
+//   every reader of its previous contents has provably finished (no barrier needed)
+// A slot is released by the completion of the last MMA that reads it, so its refill starts early.
+constexpr uint32_t ST_KQ = 0, ST_W = 32768, ST_P = 49152;
+constexpr uint32_t STAGE_A = 57344, STAGE_A_TX = 32768 + 16384 + 8192 + 1280;   // + the gate vectors
+constexpr uint32_t ST_V = 0, ST_T2 = 16384;
+constexpr uint32_t STAGE_B = 24576, STAGE_B_TX = 16384 + 8192;
+constexpr uint32_t CS_A = 0, CS_B = 2 * STAGE_A, CS_GATES = CS_B + 3 * STAGE_B;
+constexpr uint32_t CS_OST = CS_GATES + 4 * 1280;       // bf16 output staging [64][128]
 constexpr uint32_t CS_BARS = CS_OST + 16384;
-constexpr uint32_t CS_MISC = CS_BARS + 16 * 8;
+constexpr uint32_t CS_MISC = CS_BARS + 24 * 8;
 constexpr uint32_t CS_TOTAL = CS_MISC + 64;
 constexpr uint32_t CHAIN_SMEM = CS_TOTAL + 1024;
 
-enum CBar : uint32_t { CB_FULL0 = 0, CB_FULL1, CB_FREE0, CB_FREE1, CB_V, CB_S, CB_O, CB_SREADY, CB_VREADY, CB_OFREE };
+enum CBar : uint32_t { CB_FULLA0 = 0, CB_FREEA0 = 2, CB_FULLB0 = 4, CB_FREEB0 = 7, CB_V = 10, CB_S, CB_O, CB_SREADY, CB_VREADY, CB_OFREE,
+                       CB_U, CB_O1 };
 
 struct ChainParams {
     const float* s0;          // [N,H,d_k,d_v] or nullptr
@@ -490,10 +509,12 @@ struct ChainParams {
     const int32_t* cu;
     const uint8_t* items;
     const float* seg_sin;     // [B*nseg, H, d_k, d_v] incoming states of segments 1.. (sequence split), or nullptr
+    float* dbg;               // debug build: time stamps of CTA (0,0,0), [role][chunk < 32][event < 8], ns
     int B, T, H, dv;
     int nseg, seg_chunks;     // segments per sequence (1 = no split) and chunks per segment
 };
 
+template <bool DBG>
 __global__ void __launch_bounds__(CHAIN_THREADS, 1)
 gdn_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                  const __grid_constant__ CUtensorMap map_v, ChainParams p) {
@@ -516,8 +537,9 @@ gdn_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     const long slot0 = slot_base(sq.tok0, n) + cbeg;
 
     if (tid == 0) {
-        mbar_init(w.bar(CB_FULL0), 1); mbar_init(w.bar(CB_FULL1), 1);
-        mbar_init(w.bar(CB_FREE0), 257); mbar_init(w.bar(CB_FREE1), 257);   // MMA commit + chain + epilogue threads
+        for (uint32_t i = 0; i < 2; ++i) { mbar_init(w.bar(CB_FULLA0 + i), 1); mbar_init(w.bar(CB_FREEA0 + i), 2); }   // both issuers
+        mbar_init(w.bar(CB_U), 1); mbar_init(w.bar(CB_O1), 1);
+        for (uint32_t i = 0; i < 3; ++i) { mbar_init(w.bar(CB_FULLB0 + i), 1); mbar_init(w.bar(CB_FREEB0 + i), 1); }
         mbar_init(w.bar(CB_V), 1); mbar_init(w.bar(CB_S), 1); mbar_init(w.bar(CB_O), 1);
         mbar_init(w.bar(CB_SREADY), 128); mbar_init(w.bar(CB_VREADY), 128); mbar_init(w.bar(CB_OFREE), 128);
         sMisc[1] = 0;
@@ -531,6 +553,11 @@ gdn_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem = sMisc[0];
+    const unsigned long long t_start = DBG ? globaltimer_ns() : 0ull;
+    auto stamp = [&](int role, int c, int ev) {
+        if (DBG && p.dbg && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && c < 32)
+            p.dbg[(role * 32 + c) * 8 + ev] = (float)(globaltimer_ns() - t_start);
+    };
     const size_t state_off = ((size_t)n * H + h) * DK * dv + (size_t)dvb * DVB;
     const float* s_in = (seg == 0) ? (p.s0 ? p.s0 + state_off : nullptr)
                                    : p.seg_sin + ((size_t)(n * p.nseg + seg) * H + h) * DK * dv + (size_t)dvb * DVB;
@@ -561,48 +588,70 @@ gdn_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             mbar_arrive(w.bar(CB_SREADY));
         }
         for (int c = 0; c < nchunks; ++c) {
-            const uint32_t s = c & 1;
-            const float* gates = reinterpret_cast<const float*>(sm + s * STAGE_BYTES + ST_GATES);
-            w.wait(CB_V, c & 1);
+            const float* gates = reinterpret_cast<const float*>(sm + CS_GATES + (c & 3) * 1280);
+            w.wait_hot(CB_V, c & 1);
+            if (c > 0) w.wait_hot(CB_O, (c - 1) & 1);     // O2 of the previous chunk no longer reads bf16 v_new
             tc_fence_after_sync();
-#pragma unroll
-            for (int hh = 0; hh < 2; ++hh) {
-                uint32_t x[32];
-                tmem_ld32(tmem + lane_base + TM_DV + 32 * hh, x);
+            if (tid == 0) stamp(0, c, 0);
+            {
+                // v_new^T: the load of the second half is in flight while the first is converted
+                uint32_t xa[32], xb[32];
+                tmem_ld32(tmem + lane_base + TM_DV, xa);
                 tmem_wait_ld();
+                tmem_ld32(tmem + lane_base + TM_DV + 32, xb);
                 uint32_t pv[16], pd[16];
 #pragma unroll
                 for (int i = 0; i < 16; ++i) {
-                    const float v0 = __uint_as_float(x[2 * i]), v1 = __uint_as_float(x[2 * i + 1]);
-                    const float2 dec = *reinterpret_cast<const float2*>(gates + 192 + 32 * hh + 2 * i);
+                    const float v0 = __uint_as_float(xa[2 * i]), v1 = __uint_as_float(xa[2 * i + 1]);
+                    const float2 dec = *reinterpret_cast<const float2*>(gates + 192 + 2 * i);
                     pv[i] = pack_bf16(v0, v1);
                     pd[i] = pack_bf16(v0 * dec.x, v1 * dec.y);
                 }
-                tmem_st16(tmem + lane_base + TM_V + 16 * hh, pv);
-                tmem_st16(tmem + lane_base + TM_VT + 16 * hh, pd);
+                tmem_st16(tmem + lane_base + TM_V, pv);
+                tmem_st16(tmem + lane_base + TM_VT, pd);
+                tmem_wait_ld();
+#pragma unroll
+                for (int i = 0; i < 16; ++i) {
+                    const float v0 = __uint_as_float(xb[2 * i]), v1 = __uint_as_float(xb[2 * i + 1]);
+                    const float2 dec = *reinterpret_cast<const float2*>(gates + 224 + 2 * i);
+                    pv[i] = pack_bf16(v0, v1);
+                    pd[i] = pack_bf16(v0 * dec.x, v1 * dec.y);
+                }
+                tmem_st16(tmem + lane_base + TM_V + 16, pv);
+                tmem_st16(tmem + lane_base + TM_VT + 16, pd);
             }
             tmem_wait_st();
             tc_fence_before_sync();
             mbar_arrive(w.bar(CB_VREADY));
-            w.wait(CB_S, c & 1);
+            if (tid == 0) stamp(0, c, 1);
+            w.wait_hot(CB_S, c & 1);
+            w.wait_hot(CB_O1, c & 1);                      // O1 of this chunk no longer reads the bf16 state
             tc_fence_after_sync();
+            if (tid == 0) stamp(0, c, 2);
             const float gamma = gates[256];
-            mbar_arrive(w.bar(CB_FREE0 + s));          // last read of this stage by this thread
-#pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                uint32_t d[32];
-                tmem_ld32(tmem + lane_base + TM_DS + 32 * q, d);
+            {
+                // S^T <- e^{gC} S^T + dS^T, 32 columns at a time, the next load always in flight
+                uint32_t da[32], db[32];
+                tmem_ld32(tmem + lane_base + TM_DS, da);
                 tmem_wait_ld();
-                uint32_t pk[16];
 #pragma unroll
-                for (int i = 0; i < 32; ++i) S[32 * q + i] = fmaf(gamma, S[32 * q + i], __uint_as_float(d[i]));
+                for (int q = 0; q < 4; ++q) {
+                    uint32_t (&cur)[32] = (q & 1) ? db : da;
+                    uint32_t (&nxt)[32] = (q & 1) ? da : db;
+                    if (q < 3) tmem_ld32(tmem + lane_base + TM_DS + 32 * (q + 1), nxt);
+                    uint32_t pk[16];
 #pragma unroll
-                for (int i = 0; i < 16; ++i) pk[i] = pack_bf16(S[32 * q + 2 * i], S[32 * q + 2 * i + 1]);
-                tmem_st16(tmem + lane_base + TM_SBF + 16 * q, pk);
+                    for (int i = 0; i < 32; ++i) S[32 * q + i] = fmaf(gamma, S[32 * q + i], __uint_as_float(cur[i]));
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) pk[i] = pack_bf16(S[32 * q + 2 * i], S[32 * q + 2 * i + 1]);
+                    tmem_st16(tmem + lane_base + TM_SBF + 16 * q, pk);
+                    if (q < 3) tmem_wait_ld();
+                }
             }
             tmem_wait_st();
             tc_fence_before_sync();
             mbar_arrive(w.bar(CB_SREADY));
+            if (tid == 0) stamp(0, c, 3);
         }
         if (p.sT && seg == p.nseg - 1) {
 #pragma unroll
@@ -610,34 +659,31 @@ gdn_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         }
     } else if (warp < 8) {
         // =============================== epilogue warpgroup ===============================
-        setmaxnreg_dec<96>();
         const int j = tid - 128, we = j >> 5;
         const uint32_t lane_base = (uint32_t)(we * 32) << 16;
         __nv_bfloat16* ost = reinterpret_cast<__nv_bfloat16*>(sm + CS_OST);
         for (int c = 0; c < nchunks; ++c) {
-            const uint32_t s = c & 1;
             const int R = min(C, len - c * C);
-            const float* gates = reinterpret_cast<const float*>(sm + s * STAGE_BYTES + ST_GATES);
-            w.wait(CB_O, c & 1);
+            const float* gates = reinterpret_cast<const float*>(sm + CS_GATES + (c & 3) * 1280);
+            w.wait_hot(CB_O, c & 1);
             tc_fence_after_sync();
+            // take both accumulators out of tensor memory first and hand them back at once: the next
+            // chunk's output MMAs wait for this
+            uint32_t o1a[32], o1b[32], o2a[32], o2b[32];
+            tmem_ld32(tmem + lane_base + TM_O1, o1a);
+            tmem_ld32(tmem + lane_base + TM_O1 + 32, o1b);
+            tmem_ld32(tmem + lane_base + TM_O2, o2a);
+            tmem_ld32(tmem + lane_base + TM_O2 + 32, o2b);
+            tmem_wait_ld();
+            tc_fence_before_sync();
+            mbar_arrive(w.bar(CB_OFREE));
 #pragma unroll
-            for (int hh = 0; hh < 2; ++hh) {
-                uint32_t o1[32], o2[32];
-                tmem_ld32(tmem + lane_base + TM_O1 + 32 * hh, o1);
-                tmem_ld32(tmem + lane_base + TM_O2 + 32 * hh, o2);
-                tmem_wait_ld();
-                if (hh == 1) {
-                    tc_fence_before_sync();
-                    mbar_arrive(w.bar(CB_OFREE));
-                }
-#pragma unroll
-                for (int i = 0; i < 32; ++i) {
-                    const int r = 32 * hh + i;
-                    const float o = fmaf(gates[128 + r], __uint_as_float(o1[i]), __uint_as_float(o2[i]));
-                    ost[r * DVB + j] = __float2bfloat16_rn(o);
-                }
+            for (int i = 0; i < 32; ++i) {
+                const float oa = fmaf(gates[128 + i], __uint_as_float(o1a[i]), __uint_as_float(o2a[i]));
+                const float ob = fmaf(gates[160 + i], __uint_as_float(o1b[i]), __uint_as_float(o2b[i]));
+                ost[i * DVB + j] = __float2bfloat16_rn(oa);           // transpose through shared memory
+                ost[(32 + i) * DVB + j] = __float2bfloat16_rn(ob);
             }
-            mbar_arrive(w.bar(CB_FREE0 + s));          // gate vectors of this stage no longer needed
             named_bar_sync(2, 128);
             {
                 __nv_bfloat16* obase = p.out + ((size_t)(tok0 + c * C) * H + h) * dv + (size_t)dvb * DVB;
@@ -656,46 +702,64 @@ gdn_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         // =============================== control warpgroup ===============================
         setmaxnreg_dec<56>();
         if (warp == 8 && lane == 0) {
-            // ---- MMA issuer ----
-            auto issue_U = [&](uint32_t s) {
-                const uint32_t vb = base + s * STAGE_BYTES + ST_V, t2 = base + s * STAGE_BYTES + ST_T2;
-#pragma unroll
-                for (uint32_t ks = 0; ks < 4; ++ks)
-                    mma_ss(tmem + TM_DV, make_smem_desc(vb + ks * 2048, 8192, 1024),
-                           make_smem_desc(t2 + ks * 2048, 1024, 1024), ID_WU, ks > 0);
-            };
-            if (nchunks > 0) {
-                w.wait(CB_FULL0, 0);
-                issue_U(0);
-            }
+            // ---- MMA issuer of the sequential chain: v_new and the state update, nothing else ----
+            // (issuing costs tens of nanoseconds per instruction; everything off the chain is
+            //  issued by a second thread so that it does not sit between two dependent steps)
             for (int c = 0; c < nchunks; ++c) {
-                const uint32_t s = c & 1, sb = base + s * STAGE_BYTES;
-                w.wait(CB_SREADY, c & 1);
+                const uint32_t s = c & 1, sb = base + CS_A + s * STAGE_A;
+                w.wait_hot(CB_SREADY, c & 1);
+                w.wait_hot(CB_FULLA0 + s, (c >> 1) & 1);
+                w.wait_hot(CB_U, c & 1);                       // U^T of this chunk is in the accumulator
                 tc_fence_after_sync();
+                stamp(1, c, 0);
 #pragma unroll
                 for (uint32_t ks = 0; ks < 8; ++ks)            // v^T = U^T - S^T W^T
                     mma_ts(tmem + TM_DV, tmem + TM_SBF + ks * 8, make_smem_desc(sb + ST_W + ks * 2048, 1024, 1024), ID_1, 1);
                 mma_commit(w.bar(CB_V));
-                if (c > 0) { w.wait(CB_OFREE, (c - 1) & 1); tc_fence_after_sync(); }
-#pragma unroll
-                for (uint32_t ks = 0; ks < 8; ++ks)            // O1^T = S^T Q^T
-                    mma_ts(tmem + TM_O1, tmem + TM_SBF + ks * 8,
-                           make_smem_desc(sb + ST_KQ + 8192 + (ks >> 2) * 16384 + (ks & 3) * 32, 16, 1024), ID_O, ks > 0);
-                w.wait(CB_VREADY, c & 1);
+                stamp(1, c, 1);
+                w.wait_hot(CB_VREADY, c & 1);
                 tc_fence_after_sync();
+                stamp(1, c, 3);
 #pragma unroll
                 for (uint32_t ks = 0; ks < 4; ++ks)            // dS^T = (v e^{gC-g})^T K
                     mma_ts(tmem + TM_DS, tmem + TM_VT + ks * 8, make_smem_desc(sb + ST_KQ + ks * 2048, 16384, 1024), ID_2, ks > 0);
                 mma_commit(w.bar(CB_S));
+                mma_commit(w.bar(CB_FREEA0 + s));
+                stamp(1, c, 4);
+            }
+        } else if (warp == 10 && lane == 0) {
+            // ---- MMA issuer of everything off the chain: U^T, O1^T, O2^T ----
+            auto issue_U = [&](int c) {                         // U^T = V^T (T diag(b))^T of chunk c
+                const uint32_t sB = c % 3, bb = base + CS_B + sB * STAGE_B;
+                w.wait(CB_FULLB0 + sB, (c / 3) & 1);
+#pragma unroll
+                for (uint32_t ks = 0; ks < 4; ++ks)
+                    mma_ss(tmem + TM_DV, make_smem_desc(bb + ST_V + ks * 2048, 8192, 1024),
+                           make_smem_desc(bb + ST_T2 + ks * 2048, 1024, 1024), ID_WU, ks > 0);
+                mma_commit(w.bar(CB_FREEB0 + sB));
+                mma_commit(w.bar(CB_U));
+            };
+            if (nchunks > 0) issue_U(0);
+            for (int c = 0; c < nchunks; ++c) {
+                const uint32_t s = c & 1, sb = base + CS_A + s * STAGE_A;
+                w.wait(CB_SREADY, c & 1);
+                w.wait(CB_FULLA0 + s, (c >> 1) & 1);
+                if (c > 0) w.wait(CB_OFREE, (c - 1) & 1);      // the epilogue has read the previous O1, O2
+                w.wait_hot(CB_V, c & 1);                       // stay out of the tensor pipe until v_new is done
+                tc_fence_after_sync();
+#pragma unroll
+                for (uint32_t ks = 0; ks < 8; ++ks)            // O1^T = S^T Q^T
+                    mma_ts(tmem + TM_O1, tmem + TM_SBF + ks * 8,
+                           make_smem_desc(sb + ST_KQ + 8192 + (ks >> 2) * 16384 + (ks & 3) * 32, 16, 1024), ID_O, ks > 0);
+                mma_commit(w.bar(CB_O1));
+                w.wait(CB_VREADY, c & 1);
+                tc_fence_after_sync();
+                if (c + 1 < nchunks) issue_U(c + 1);           // D_v is free: v_new of chunk c has been read
 #pragma unroll
                 for (uint32_t ks = 0; ks < 4; ++ks)            // O2^T = v^T P^T
                     mma_ts(tmem + TM_O2, tmem + TM_V + ks * 8, make_smem_desc(sb + ST_P + ks * 32, 16, 1024), ID_O, ks > 0);
                 mma_commit(w.bar(CB_O));
-                mma_commit(w.bar(CB_FREE0 + s));
-                if (c + 1 < nchunks) {
-                    w.wait(CB_FULL0 + ((c + 1) & 1), ((c + 1) >> 1) & 1);
-                    issue_U((c + 1) & 1);                      // D_v is free: v_new of chunk c has been read
-                }
+                mma_commit(w.bar(CB_FREEA0 + s));
             }
         } else if (warp == 9 && lane == 0) {
             // ---- TMA producer ----
@@ -703,28 +767,36 @@ gdn_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             prefetch_tensormap(&map_k);
             prefetch_tensormap(&map_v);
             for (int c = 0; c < nchunks; ++c) {
-                const uint32_t s = c & 1, sb = base + s * STAGE_BYTES;
-                if (c >= 2) w.wait(CB_FREE0 + s, ((c - 2) >> 1) & 1);
-                const uint32_t full = w.bar(CB_FULL0 + s);
                 const int tok = (int)(tok0 + (long)c * C);
                 const uint8_t* item = p.items + (size_t)((slot0 + c) * H + h) * ITEM_BYTES;
-                mbar_arrive_expect_tx(full, STAGE_TX);
-                tma_load_3d(sb + ST_KQ, &map_k, 0, h, tok, full);
-                tma_load_3d(sb + ST_KQ + 8192, &map_q, 0, h, tok, full);
-                tma_load_3d(sb + ST_KQ + 16384, &map_k, 64, h, tok, full);
-                tma_load_3d(sb + ST_KQ + 24576, &map_q, 64, h, tok, full);
-                tma_load_3d(sb + ST_V, &map_v, dvb * DVB, h, tok, full);
-                tma_load_3d(sb + ST_V + 8192, &map_v, dvb * DVB + 64, h, tok, full);
-                bulk_load(sb + ST_W, item + IT_W, 16384, full);
-                bulk_load(sb + ST_T2, item + IT_T2, 8192, full);
-                bulk_load(sb + ST_P, item + IT_P, 8192, full);
-                bulk_load(sb + ST_GATES, item + IT_GATES, 1280, full);
+                {   // ring B: V tile and (T diag(b))^T
+                    const uint32_t sB = c % 3, bb = base + CS_B + sB * STAGE_B, full = w.bar(CB_FULLB0 + sB);
+                    if (c >= 3) w.wait(CB_FREEB0 + sB, ((c / 3) - 1) & 1);
+                    mbar_arrive_expect_tx(full, STAGE_B_TX);
+                    tma_load_3d(bb + ST_V, &map_v, dvb * DVB, h, tok, full);
+                    tma_load_3d(bb + ST_V + 8192, &map_v, dvb * DVB + 64, h, tok, full);
+                    bulk_load(bb + ST_T2, item + IT_T2, 8192, full);
+                }
+                {   // ring A: K/Q tiles, -W^T, P, and the gate vectors (own 4-deep ring, same barrier)
+                    const uint32_t s = c & 1, sb = base + CS_A + s * STAGE_A, full = w.bar(CB_FULLA0 + s);
+                    if (c >= 2) w.wait(CB_FREEA0 + s, ((c >> 1) - 1) & 1);
+                    mbar_arrive_expect_tx(full, STAGE_A_TX);
+                    bulk_load(sb + ST_W, item + IT_W, 16384, full);
+                    tma_load_3d(sb + ST_KQ, &map_k, 0, h, tok, full);
+                    tma_load_3d(sb + ST_KQ + 8192, &map_q, 0, h, tok, full);
+                    tma_load_3d(sb + ST_KQ + 16384, &map_k, 64, h, tok, full);
+                    tma_load_3d(sb + ST_KQ + 24576, &map_q, 64, h, tok, full);
+                    bulk_load(sb + ST_P, item + IT_P, 8192, full);
+                    bulk_load(base + CS_GATES + (c & 3) * 1280, item + IT_GATES, 1280, full);
+                }
             }
             if (*w.abort_flag) {
-                for (int c = max(0, nchunks - 2); c < nchunks; ++c) {
-                    const uint32_t bar = w.bar(CB_FULL0 + (c & 1));
-                    const unsigned long long t0 = globaltimer_ns();
-                    while (!mbar_try_wait(bar, (c >> 1) & 1) && globaltimer_ns() - t0 < TIMEOUT_NS) {}
+                // let copies in flight land before shared memory is released (bounded)
+                const unsigned long long t0 = globaltimer_ns();
+                for (int c = max(0, nchunks - 3); c < nchunks; ++c) {
+                    while (!mbar_try_wait(w.bar(CB_FULLB0 + c % 3), (c / 3) & 1) && globaltimer_ns() - t0 < TIMEOUT_NS) {}
+                    if (c >= nchunks - 2)
+                        while (!mbar_try_wait(w.bar(CB_FULLA0 + (c & 1)), (c >> 1) & 1) && globaltimer_ns() - t0 < TIMEOUT_NS) {}
                 }
             }
         }
@@ -1118,7 +1190,8 @@ int launch_lean(const PrefillArgs& a, void* workspace, size_t workspace_bytes, c
             return GDN_ERR_CUDA;
     }
     if (cudaFuncSetAttribute(gdn_prep_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)PREP_SMEM) != cudaSuccess ||
-        cudaFuncSetAttribute(gdn_chain_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)CHAIN_SMEM) != cudaSuccess ||
+        cudaFuncSetAttribute(gdn_chain_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)CHAIN_SMEM) != cudaSuccess ||
+        cudaFuncSetAttribute(gdn_chain_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)CHAIN_SMEM) != cudaSuccess ||
         cudaFuncSetAttribute(gdn_summary_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SUM_SMEM) != cudaSuccess ||
         cudaFuncSetAttribute(gdn_combine_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)CMB_SMEM) != cudaSuccess)
         return GDN_ERR_CUDA;
@@ -1167,15 +1240,17 @@ int launch_lean(const PrefillArgs& a, void* workspace, size_t workspace_bytes, c
     g_lean_split_last = nseg > 1;
     // ---- steps c, d ----
     ChainParams cp{a.initial_state, static_cast<__nv_bfloat16*>(a.out), a.final_state, a.cu_seqlens,
-                   ws, seg_sin, a.B, a.T, a.H, a.d_v, nseg, seg_chunks};
+                   ws, seg_sin, g_lean_dbg, a.B, a.T, a.H, a.d_v, nseg, seg_chunks};
     dim3 grid(a.d_v / DVB, a.H, a.B * nseg);
-    gdn_chain_kernel<<<grid, CHAIN_THREADS, CHAIN_SMEM, stream>>>(mq, mk, mv, cp);
+    if (g_lean_dbg) gdn_chain_kernel<true><<<grid, CHAIN_THREADS, CHAIN_SMEM, stream>>>(mq, mk, mv, cp);
+    else gdn_chain_kernel<false><<<grid, CHAIN_THREADS, CHAIN_SMEM, stream>>>(mq, mk, mv, cp);
     count_launch();
     mark(4);
     return cudaGetLastError() == cudaSuccess ? GDN_OK : GDN_ERR_CUDA;
 }
 
 void lean_force_segments(int nseg) { g_lean_force_nseg = nseg; }
+void lean_set_debug(float* p) { g_lean_dbg = p; }
 
 int lean_set_timing(int enable) {
     if (enable)
@@ -1243,7 +1318,7 @@ int launch_lean_static(const PrefillArgs& a, cudaStream_t stream) {
         if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
             return GDN_ERR_CUDA;
         if (cudaFuncSetAttribute(gdn_prep_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)PREP_SMEM) != cudaSuccess ||
-            cudaFuncSetAttribute(gdn_chain_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)CHAIN_SMEM) != cudaSuccess)
+            cudaFuncSetAttribute(gdn_chain_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)CHAIN_SMEM) != cudaSuccess)
             return GDN_ERR_CUDA;
         sms_of_device[dev] = sms;
         scratch_of_device[dev] = ptr;
@@ -1261,9 +1336,9 @@ int launch_lean_static(const PrefillArgs& a, cudaStream_t stream) {
     if (cudaGetLastError() != cudaSuccess) return GDN_ERR_CUDA;
     const int nch = packed ? 1 : (a.T + C - 1) / C;            // one segment: the whole sequence
     ChainParams cp{a.initial_state, static_cast<__nv_bfloat16*>(a.out), a.final_state, a.cu_seqlens,
-                   ws, nullptr, a.B, a.T, a.H, a.d_v, 1, packed ? (1 << 24) : (nch > 0 ? nch : 1)};
+                   ws, nullptr, nullptr, a.B, a.T, a.H, a.d_v, 1, packed ? (1 << 24) : (nch > 0 ? nch : 1)};
     dim3 grid(a.d_v / DVB, a.H, a.B);
-    gdn_chain_kernel<<<grid, CHAIN_THREADS, CHAIN_SMEM, stream>>>(mq, mk, mv, cp);
+    gdn_chain_kernel<false><<<grid, CHAIN_THREADS, CHAIN_SMEM, stream>>>(mq, mk, mv, cp);
     count_launch();
     return cudaGetLastError() == cudaSuccess ? GDN_OK : GDN_ERR_CUDA;
 }
