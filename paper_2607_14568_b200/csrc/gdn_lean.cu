@@ -5,7 +5,7 @@
 // sits, once per chunk, on one warpgroup of the few SMs that own a (sequence, head) chain.
 // Here everything that does not depend on the incoming state is taken off those SMs:
 //
-//   gdn_prep_kernel    grid over every (chunk, head), all SMs, two CTAs per SM:
+//   gdn_prep_kernel    grid over every (chunk, head), all SMs, three CTAs per SM:
 //                      step a  cumulative log gate and the gate vectors,
 //                      step b1 G = [K;Q] K^T on the tensor core, decay masks -> A (fp32), P (bf16),
 //                      step b2 T = (I + A)^{-1}, blocked forward substitution in shared memory,
@@ -121,8 +121,8 @@ __device__ __forceinline__ SeqInfo seq_info(const int32_t* cu, int n, int T) {
 // prepare kernel
 // =====================================================================================
 constexpr uint32_t PS_KQ = 0;                         // [K_lo | Q_lo | K_hi | Q_hi]
-constexpr uint32_t PS_T1 = 32768;                     // (T diag(b e^g))^T image
-constexpr uint32_t PS_A = PS_T1 + 8192;
+constexpr uint32_t PS_A = 32768;                      // fp32 A [64][68] ...
+constexpr uint32_t PS_T1 = PS_A;                      // ... whose space later holds the (T diag(b e^g))^T image
 constexpr uint32_t PS_TF = PS_A + 64 * LDA * 4;
 constexpr uint32_t PS_Y = PS_TF + 64 * LDA * 4;
 constexpr uint32_t PS_GATES = PS_Y + 32 * LDY * 4;
@@ -150,7 +150,7 @@ constexpr uint32_t ID_1 = make_idesc(128, 64, kFmtBF16, kFmtBF16, kMajorK, kMajo
 constexpr uint32_t ID_O = make_idesc(128, 64, kFmtBF16, kFmtBF16, kMajorK, kMajorK);
 constexpr uint32_t ID_2 = make_idesc(128, 128, kFmtBF16, kFmtBF16, kMajorK, kMajorMN);
 
-__global__ void __launch_bounds__(PREP_THREADS, 2)
+__global__ void __launch_bounds__(PREP_THREADS, 3)
 gdn_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k, PrepParams p) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -875,7 +875,7 @@ gdn_summary_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
     if (tid == 0) {
         for (uint32_t i = 0; i < SUM_STAGES; ++i) {
             mbar_init(w.bar(SB_FULL0 + i), 1);
-            mbar_init(w.bar(SB_FREE0 + i), 1 + 128 * ninst);
+            mbar_init(w.bar(SB_FREE0 + i), 129 * ninst);         // per instance: its issue thread and its warpgroup
         }
         for (uint32_t i = 0; i < 2; ++i) {
             mbar_init(w.bar(SB_V0 + i), 1); mbar_init(w.bar(SB_S0 + i), 1);
@@ -918,7 +918,7 @@ gdn_summary_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
             for (int c = 0; c < nchunks; ++c) {
                 const uint32_t s = c % SUM_STAGES;
                 const float* gates = reinterpret_cast<const float*>(sm + s * SUM_STAGE + SS_GATES);
-                w.wait(SB_V0 + inst, c & 1);
+                w.wait_hot(SB_V0 + inst, c & 1);
                 tc_fence_after_sync();
 #pragma unroll
                 for (int hh = 0; hh < 2; ++hh) {
@@ -936,7 +936,7 @@ gdn_summary_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
                 tmem_wait_st();
                 tc_fence_before_sync();
                 mbar_arrive(w.bar(SB_VREADY0 + inst));
-                w.wait(SB_S0 + inst, c & 1);
+                w.wait_hot(SB_S0 + inst, c & 1);
                 tc_fence_after_sync();
                 const float gamma = gates[256];
                 mbar_arrive(w.bar(SB_FREE0 + s));
@@ -970,34 +970,36 @@ gdn_summary_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
     } else {
         // =============================== control warpgroup ===============================
         setmaxnreg_dec<56>();
-        if (warp == 8 && lane == 0) {
-            for (int c = 0; c < nchunks; ++c) {
-                const uint32_t s = c % SUM_STAGES, sb = base + s * SUM_STAGE;
-                w.wait(SB_FULL0 + s, (c / SUM_STAGES) & 1);
-                tc_fence_after_sync();
+        if ((warp == 8 || warp == 10) && lane == 0) {
+            // ---- one MMA issue thread per chain instance (they are independent) ----
+            const int inst = (warp == 8) ? 0 : 1;
+            if (inst < ninst) {
+                for (int c = 0; c < nchunks; ++c) {
+                    const uint32_t s = c % SUM_STAGES, sb = base + s * SUM_STAGE;
+                    w.wait_hot(SB_FULL0 + s, (c / SUM_STAGES) & 1);
+                    if (inst == 0) {
+                        tc_fence_after_sync();
 #pragma unroll
-                for (uint32_t ks = 0; ks < 4; ++ks)            // U^T = V^T (T diag(b))^T
-                    mma_ss(tmem + sum_dv(0), make_smem_desc(sb + SS_V + ks * 2048, 8192, 1024),
-                           make_smem_desc(sb + SS_T2 + ks * 2048, 1024, 1024), ID_WU, ks > 0);
-                for (int inst = 0; inst < ninst; ++inst) {
-                    w.wait(SB_SREADY0 + inst, c & 1);
+                        for (uint32_t ks = 0; ks < 4; ++ks)        // U^T = V^T (T diag(b))^T
+                            mma_ss(tmem + sum_dv(0), make_smem_desc(sb + SS_V + ks * 2048, 8192, 1024),
+                                   make_smem_desc(sb + SS_T2 + ks * 2048, 1024, 1024), ID_WU, ks > 0);
+                    }
+                    w.wait_hot(SB_SREADY0 + inst, c & 1);
                     tc_fence_after_sync();
 #pragma unroll
-                    for (uint32_t ks = 0; ks < 8; ++ks)        // v^T = U^T - S^T W^T   (U = 0 for the identity chain)
+                    for (uint32_t ks = 0; ks < 8; ++ks)            // v^T = U^T - S^T W^T   (U = 0 for the identity chain)
                         mma_ts(tmem + sum_dv(inst), tmem + sum_ds(inst) + ks * 8,
                                make_smem_desc(sb + SS_W + ks * 2048, 1024, 1024), ID_1, (inst == 0 || ks > 0) ? 1u : 0u);
                     mma_commit(w.bar(SB_V0 + inst));
-                }
-                for (int inst = 0; inst < ninst; ++inst) {
-                    w.wait(SB_VREADY0 + inst, c & 1);
+                    w.wait_hot(SB_VREADY0 + inst, c & 1);
                     tc_fence_after_sync();
 #pragma unroll
-                    for (uint32_t ks = 0; ks < 4; ++ks)        // dS^T = (v e^{gC-g})^T K
+                    for (uint32_t ks = 0; ks < 4; ++ks)            // dS^T = (v e^{gC-g})^T K
                         mma_ts(tmem + sum_ds(inst), tmem + sum_vt(inst) + ks * 8,
                                make_smem_desc(sb + SS_K + ks * 2048, 8192, 1024), ID_2, ks > 0);
                     mma_commit(w.bar(SB_S0 + inst));
+                    mma_commit(w.bar(SB_FREE0 + s));
                 }
-                mma_commit(w.bar(SB_FREE0 + s));
             }
         } else if (warp == 9 && lane == 0) {
             prefetch_tensormap(&map_k);
@@ -1200,7 +1202,7 @@ int launch_lean(const PrefillArgs& a, void* workspace, size_t workspace_bytes, c
     const long nitems = nslots * a.H;
     // ---- state-independent steps, every (chunk, head) ----
     PrepParams pp{a.log_alpha, a.beta, a.cu_seqlens, ws, nslots, a.B, a.T, a.H};
-    const int pgrid = (int)(nitems < 2L * num_sms ? nitems : 2L * num_sms);
+    const int pgrid = (int)(nitems < 3L * num_sms ? nitems : 3L * num_sms);
     auto mark = [&](int i) { if (g_lean_timing && g_lean_events[i]) cudaEventRecord(g_lean_events[i], stream); };
     mark(0);
     gdn_prep_kernel<<<pgrid, PREP_THREADS, PREP_SMEM, stream>>>(mq, mk, pp);
@@ -1329,7 +1331,7 @@ int launch_lean_static(const PrefillArgs& a, cudaStream_t stream) {
         !tc_make_map(&mv, a.v, tokens, a.H, a.d_v))
         return GDN_ERR_CUDA;
     const long nitems = (long)nslots * a.H;
-    const long cap = 2L * sms_of_device[dev];
+    const long cap = 3L * sms_of_device[dev];
     PrepParams pp{a.log_alpha, a.beta, a.cu_seqlens, ws, (long)nslots, a.B, a.T, a.H};
     gdn_prep_kernel<<<(int)(nitems < cap ? nitems : cap), PREP_THREADS, PREP_SMEM, stream>>>(mq, mk, pp);
     count_launch();
