@@ -150,6 +150,25 @@ constexpr uint32_t ID_1 = make_idesc(128, 64, kFmtBF16, kFmtBF16, kMajorK, kMajo
 constexpr uint32_t ID_O = make_idesc(128, 64, kFmtBF16, kFmtBF16, kMajorK, kMajorK);
 constexpr uint32_t ID_2 = make_idesc(128, 128, kFmtBF16, kFmtBF16, kMajorK, kMajorMN);
 
+// item -> (head, first token, valid rows); false for a slot no sequence uses
+__device__ __forceinline__ bool decode_item(const PrepParams& p, long item, int* h, long* tok, int* R) {
+    const long slot = item / p.H;
+    *h = (int)(item - slot * p.H);
+    // which sequence owns this slot?  (largest n with slot_base(n) <= slot)
+    int lo = 0, hi = p.B - 1;
+    while (lo < hi) {
+        const int mid = (lo + hi + 1) >> 1;
+        const long t0 = p.cu ? (long)p.cu[mid] : (long)mid * p.T;
+        if (slot_base(t0, mid) <= slot) lo = mid; else hi = mid - 1;
+    }
+    const SeqInfo sq = seq_info(p.cu, lo, p.T);
+    const int c = (int)(slot - slot_base(sq.tok0, lo));
+    if (c < 0 || c * C >= sq.len) return false;
+    *R = min(C, sq.len - c * C);
+    *tok = sq.tok0 + (long)c * C;
+    return true;
+}
+
 __global__ void __launch_bounds__(PREP_THREADS, 3)
 gdn_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k, PrepParams p) {
     extern __shared__ uint8_t smem_raw[];
@@ -182,30 +201,9 @@ gdn_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     const long nitems = p.nslots * H;
     int it = 0;     // items this CTA has processed (barrier phases)
     for (long item = blockIdx.x; item < nitems; item += gridDim.x) {
-        const long slot = item / H;
-        const int h = (int)(item - slot * H);
-        // which sequence owns this slot?  (largest n with slot_base(n) <= slot)
-        int n = 0;
-        if (p.cu) {
-            int lo = 0, hi = p.B - 1;
-            while (lo < hi) {
-                const int mid = (lo + hi + 1) >> 1;
-                if (slot_base(p.cu[mid], mid) <= slot) lo = mid; else hi = mid - 1;
-            }
-            n = lo;
-        } else {
-            int lo = 0, hi = p.B - 1;
-            while (lo < hi) {
-                const int mid = (lo + hi + 1) >> 1;
-                if (slot_base((long)mid * p.T, mid) <= slot) lo = mid; else hi = mid - 1;
-            }
-            n = lo;
-        }
-        const SeqInfo sq = seq_info(p.cu, n, p.T);
-        const int c = (int)(slot - slot_base(sq.tok0, n));
-        if (c * C >= sq.len) continue;                       // unused slot (uniform for the CTA)
-        const int R = min(C, sq.len - c * C);
-        const long tok = sq.tok0 + (long)c * C;
+        int h, R;
+        long tok;
+        if (!decode_item(p, item, &h, &tok, &R)) continue;   // unused slot (uniform for the CTA)
         uint8_t* out_item = p.items + (size_t)item * ITEM_BYTES;
         const uint32_t par = it & 1;
 
@@ -426,6 +424,16 @@ gdn_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                 tma_load_3d(kq + 8192, &map_q, 0, h, (int)tok, full);
                 tma_load_3d(kq + 16384, &map_k, 64, h, (int)tok, full);
                 tma_load_3d(kq + 24576, &map_q, 64, h, (int)tok, full);
+                {   // the tiles of this CTA's next item: into L2 now, so that their TMA load is short
+                    int h2, R2;
+                    long tok2;
+                    if (item + gridDim.x < nitems && decode_item(p, item + gridDim.x, &h2, &tok2, &R2)) {
+                        tma_prefetch_3d(&map_k, 0, h2, (int)tok2);
+                        tma_prefetch_3d(&map_q, 0, h2, (int)tok2);
+                        tma_prefetch_3d(&map_k, 64, h2, (int)tok2);
+                        tma_prefetch_3d(&map_q, 64, h2, (int)tok2);
+                    }
+                }
                 w.wait(PB_FULL, par);
 #pragma unroll
                 for (uint32_t ks = 0; ks < 8; ++ks) {
@@ -1044,7 +1052,8 @@ constexpr int CMB_THREADS = 512;                       // 4 groups along the con
 constexpr uint32_t CMB_MT_BYTES = DK * DK * 4;
 constexpr uint32_t CMB_BUFS = 2;
 constexpr uint32_t CMB_S_BYTES = DK * CMB_COLS * 4;
-constexpr uint32_t CMB_SMEM = CMB_BUFS * CMB_MT_BYTES + 5 * CMB_S_BYTES + 64 + 128;
+constexpr int CMB_LDP = CMB_COLS + 4;                  // padded row of the partial sums (bank spread)
+constexpr uint32_t CMB_SMEM = CMB_BUFS * CMB_MT_BYTES + CMB_S_BYTES + 4 * DK * CMB_LDP * 4 + 64 + 128;
 struct CombineParams {
     const float* s0;          // [B, H, d_k, d_v] or nullptr
     const float* seg_n;
@@ -1060,14 +1069,15 @@ __global__ void __launch_bounds__(CMB_THREADS) gdn_combine_kernel(CombineParams 
     const float* sMt = reinterpret_cast<const float*>(sm);                                   // [CMB_BUFS][i][m]
     float (*sS)[CMB_COLS] = reinterpret_cast<float (*)[CMB_COLS]>(sm + CMB_BUFS * CMB_MT_BYTES);
     float* sPart = reinterpret_cast<float*>(sm + CMB_BUFS * CMB_MT_BYTES + CMB_S_BYTES);     // [4][m][16]
-    const uint32_t misc = CMB_BUFS * CMB_MT_BYTES + 5 * CMB_S_BYTES;
+    const uint32_t misc = CMB_BUFS * CMB_MT_BYTES + CMB_S_BYTES + 4 * DK * CMB_LDP * 4;
     volatile int* abort_flag = reinterpret_cast<volatile int*>(sm + misc + 32);
     Waiter w{base + misc, abort_flag};
 
     const int tid = threadIdx.x;
     const int j0 = blockIdx.x * CMB_COLS, h = blockIdx.y, n = blockIdx.z;
     const int H = p.H, dv = p.dv;
-    const int kg = tid >> 7, mt4 = tid & 31, ct = (tid >> 5) & 3;     // product phase
+    // product phase: a warp covers 8 row tiles x 4 column tiles, so its M loads touch one 128-byte line
+    const int kg = tid >> 7, ct = tid & 3, mt4 = ((tid >> 2) & 7) + 8 * ((tid >> 5) & 3);
     const int rm = tid >> 2, rc = (tid & 3) * 4;                       // reduction phase: 4 outputs of row rm
     auto load_mt = [&](int seg) {
         const uint32_t buf = seg % CMB_BUFS, full = w.bar(buf);
@@ -1117,14 +1127,14 @@ __global__ void __launch_bounds__(CMB_THREADS) gdn_combine_kernel(CombineParams 
         }
 #pragma unroll
         for (int r = 0; r < 4; ++r)
-            *reinterpret_cast<float4*>(sPart + (kg * DK + 4 * mt4 + r) * CMB_COLS + 4 * ct) =
+            *reinterpret_cast<float4*>(sPart + (kg * DK + 4 * mt4 + r) * CMB_LDP + 4 * ct) =
                 make_float4(acc[r][0], acc[r][1], acc[r][2], acc[r][3]);
         __syncthreads();                               // partial products done; sS and this M buffer are free
         if (tid == 0 && seg + (int)CMB_BUFS < p.nseg - 1) load_mt(seg + CMB_BUFS);
         float4 o = ncur;
 #pragma unroll
         for (int g = 0; g < 4; ++g) {
-            const float4 q = *reinterpret_cast<const float4*>(sPart + (g * DK + rm) * CMB_COLS + rc);
+            const float4 q = *reinterpret_cast<const float4*>(sPart + (g * DK + rm) * CMB_LDP + rc);
             o.x += q.x; o.y += q.y; o.z += q.z; o.w += q.w;
         }
         *reinterpret_cast<float4*>(&sS[rm][rc]) = o;
