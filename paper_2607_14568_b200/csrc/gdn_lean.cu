@@ -424,16 +424,6 @@ gdn_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                 tma_load_3d(kq + 8192, &map_q, 0, h, (int)tok, full);
                 tma_load_3d(kq + 16384, &map_k, 64, h, (int)tok, full);
                 tma_load_3d(kq + 24576, &map_q, 64, h, (int)tok, full);
-                {   // the tiles of this CTA's next item: into L2 now, so that their TMA load is short
-                    int h2, R2;
-                    long tok2;
-                    if (item + gridDim.x < nitems && decode_item(p, item + gridDim.x, &h2, &tok2, &R2)) {
-                        tma_prefetch_3d(&map_k, 0, h2, (int)tok2);
-                        tma_prefetch_3d(&map_q, 0, h2, (int)tok2);
-                        tma_prefetch_3d(&map_k, 64, h2, (int)tok2);
-                        tma_prefetch_3d(&map_q, 64, h2, (int)tok2);
-                    }
-                }
                 w.wait(PB_FULL, par);
 #pragma unroll
                 for (uint32_t ks = 0; ks < 8; ++ks) {
