@@ -360,6 +360,45 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+def run_decode(args):
+    """Secondary line: one decode step (state streamed once in, once out), B = 256 sequences."""
+    import torch
+
+    import paper_2607_14568_b200 as gdn
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    B, H, dk, dv = 256, 16, 128, 128
+    g = torch.Generator(device="cuda").manual_seed(0)
+    q = torch.nn.functional.normalize(torch.randn(B, H, dk, device="cuda", generator=g), dim=-1).bfloat16()
+    k = torch.nn.functional.normalize(torch.randn(B, H, dk, device="cuda", generator=g), dim=-1).bfloat16()
+    v = torch.randn(B, H, dv, device="cuda", generator=g).bfloat16()
+    la = -torch.nn.functional.softplus(torch.randn(B, H, device="cuda", generator=g)) * 0.05
+    be = torch.sigmoid(torch.randn(B, H, device="cuda", generator=g))
+    state = torch.randn(B, H, dk, dv, device="cuda", generator=g) * 0.02
+    out = torch.empty_like(v)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    for _ in range(max(args.warmup, 3)):
+        gdn.gdn_decode_step(q, k, v, la, be, state, out)
+    torch.cuda.synchronize()
+    for a, b in ev:
+        flush.fill_(1)
+        a.record()
+        gdn.gdn_decode_step(q, k, v, la, be, state, out)
+        b.record()
+    torch.cuda.synchronize()
+    ms = float(np.mean([a.elapsed_time(b) for a, b in ev]))
+    nbytes = 2 * B * H * dk * dv * 4 + B * H * ((2 * dk + 2 * dv) * 2 + 8)
+    peaks = measured_peaks()
+    gbs = nbytes / (ms * 1e-3) / 1e9
+    print(json.dumps({"metric": "gdn_decode_step_tokens_per_s", "value": B / (ms * 1e-3), "unit": "tokens/s",
+                      "n_gpus": 1, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms,
+                      "higher_is_better": True, "dtype": "f32", "data": "synthetic",
+                      "config": {"workload": "decode", "B": B, "H": H, "d_k": dk, "d_v": dv},
+                      "roofline": {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                                   "frac": gbs / peaks["hbm_gbs"], "traffic": None, "peak_source": peaks["source"],
+                                   "kernel": "gdn_decode_kernel", "algorithmic_bytes": nbytes}}), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -371,6 +410,8 @@ def main():
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.workload == "decode":
+        run_decode(args)
     else:
         run_ours(args)
 

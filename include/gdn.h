@@ -126,6 +126,21 @@ int gdn_chunk_prefill_host(const void* q_host, const void* k_host, const void* v
 size_t gdn_host_staging_bytes(int B, int T, int H, int d_k, int d_v);
 
 /*
+ * One decode step: the same recurrence for a single new token per sequence, continuing from
+ * the state a prefill returned (Section "The model": the state is "updated token-by-token";
+ * Section "Decode, and why 4-bit is slower": decode is bandwidth-bound -- here the state is
+ * read once and written once).  q, k [B, H, d_k] and v, out [B, H, d_v] are bf16; log_alpha,
+ * beta [B, H] fp32; state [B, H, d_k, d_v] fp32 is updated IN PLACE (it is both the incoming
+ * and the outgoing state).  Supported: d_k a multiple of 8 up to 128, d_v a multiple of 128.
+ * Errors as gdn_chunk_prefill; asynchronous on `stream`; allocates nothing.
+ */
+int gdn_decode_step(const void* q, const void* k, const void* v,
+                    const float* log_alpha, const float* beta,
+                    float* state, void* out,
+                    int B, int H, int d_k, int d_v,
+                    gdn_stream_t stream);
+
+/*
  * Optional scratch memory.  Without it gdn_chunk_prefill runs one fused kernel per call in
  * which each (sequence, head) chain also does its own forward substitutions.  With scratch of
  * at least gdn_workspace_bytes(...) bytes the state-independent steps (cumulative gate,

@@ -46,6 +46,8 @@ def lib():
         L.gdn_chunk_prefill_host.restype = i
         L.gdn_host_staging_bytes.argtypes = [i] * 5
         L.gdn_host_staging_bytes.restype = sz
+        L.gdn_decode_step.argtypes = [vp] * 7 + [i] * 4 + [vp]
+        L.gdn_decode_step.restype = i
         L.gdn_workspace_bytes.argtypes = [i] * 6
         L.gdn_workspace_bytes.restype = sz
         L.gdn_set_workspace.argtypes = [vp, sz]
@@ -191,6 +193,25 @@ def gdn_chunk_prefill_noalloc(q, k, v, log_alpha, beta, initial_state, out, fina
     does not fit.  Make the first call on a device outside stream capture; do not overlap calls."""
     return _prefill("gdn_chunk_prefill_noalloc", torch.bfloat16, q, k, v, log_alpha, beta, initial_state,
                     out, final_state, cu_seqlens, chunk, stream)
+
+
+def gdn_decode_step(q, k, v, log_alpha, beta, state, out, stream=None):
+    """One token per sequence: q, k [B,H,d_k], v, out [B,H,d_v] bf16; log_alpha, beta [B,H] fp32;
+    state [B,H,d_k,d_v] fp32, updated in place.  See include/gdn.h."""
+    f32, bf = torch.float32, torch.bfloat16
+    _check([("q", q, bf), ("k", k, bf), ("v", v, bf), ("out", out, bf), ("log_alpha", log_alpha, f32),
+            ("beta", beta, f32), ("state", state, f32)], bf, "cuda")
+    B, H, d_k = q.shape
+    d_v = v.shape[-1]
+    if k.shape != q.shape or tuple(v.shape) != (B, H, d_v) or out.shape != v.shape:
+        raise ValueError("q, k, v, out shapes disagree")
+    if tuple(log_alpha.shape) != (B, H) or tuple(beta.shape) != (B, H) or tuple(state.shape) != (B, H, d_k, d_v):
+        raise ValueError("gate or state shapes disagree with q, v")
+    rc = lib().gdn_decode_step(_ptr(q), _ptr(k), _ptr(v), _ptr(log_alpha), _ptr(beta), _ptr(state), _ptr(out),
+                               int(B), int(H), int(d_k), int(d_v), _stream(stream))
+    if rc != 0:
+        raise GdnError(rc, "gdn_decode_step")
+    return out, state
 
 
 def gdn_chunk_prefill_host(q, k, v, log_alpha, beta, initial_state, out, final_state, cu_seqlens,

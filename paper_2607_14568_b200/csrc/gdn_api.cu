@@ -172,6 +172,16 @@ int gdn_chunk_prefill_noalloc(const void* q, const void* k, const void* v, const
     return launch_lean_static(a, reinterpret_cast<cudaStream_t>(stream));
 }
 
+int gdn_decode_step(const void* q, const void* k, const void* v, const float* log_alpha, const float* beta,
+                    float* state, void* out, int B, int H, int d_k, int d_v, gdn_stream_t stream) {
+    if (!q || !k || !v || !log_alpha || !beta || !state || !out) return GDN_ERR_INVALID_ARG;
+    if (B <= 0 || H <= 0 || d_k <= 0 || d_v <= 0) return GDN_ERR_INVALID_ARG;
+    const void* ptrs[] = {q, k, v, log_alpha, beta, state, out};
+    for (const void* p : ptrs)
+        if (!aligned16(p)) return GDN_ERR_UNSUPPORTED;
+    return launch_decode(q, k, v, log_alpha, beta, state, out, B, H, d_k, d_v, reinterpret_cast<cudaStream_t>(stream));
+}
+
 size_t gdn_workspace_bytes(int B, int T, int H, int d_k, int d_v, int packed) {
     return lean_workspace_bytes(B, T, H, d_k, d_v, packed != 0);
 }

@@ -49,6 +49,11 @@ void lean_set_debug(float* p);        // tests only: time stamps of the chain ke
 int lean_set_timing(int enable);      // benchmark only: record events around each kernel
 int lean_get_timing(float* ms4);      // {prepare, summary, combine, chain} of the last call
 
+// Single-token decode step (bf16 q/k/v/out, fp32 state updated in place).
+bool decode_supported(int d_k, int d_v);
+int launch_decode(const void* q, const void* k, const void* v, const float* log_alpha, const float* beta,
+                  float* state, void* out, int B, int H, int d_k, int d_v, cudaStream_t stream);
+
 void count_launch(int n = 1);
 
 }  // namespace gdn
