@@ -106,6 +106,15 @@ __device__ __forceinline__ void bulk_load(uint32_t smem_dst, const void* gsrc, u
                  ::"r"(smem_dst), "l"(reinterpret_cast<uint64_t>(gsrc)), "r"(bytes), "r"(bar) : "memory");
 }
 
+// plain bulk copy shared -> global (16-byte aligned, size % 16 == 0), tracked by bulk groups
+__device__ __forceinline__ void bulk_store(void* gdst, uint32_t smem_src, uint32_t bytes) {
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
+                 ::"l"(reinterpret_cast<uint64_t>(gdst)), "r"(smem_src), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read_all() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+
 // slot of chunk 0 of sequence n: disjoint ranges for any lengths, total <= tokens/64 + B
 __device__ __forceinline__ long slot_base(long tok0, int n) { return (tok0 >> 6) + n; }
 
@@ -221,7 +230,7 @@ gdn_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                 const float br = gates[64 + r];
                 const bool is_a = tp < 64;
                 const int rmax = 32 * (warp & 1) + 31;
-                uint8_t* pimg = out_item + IT_P;
+                const uint32_t pimg = base + PS_KQ + 8192;   // the Q_lo sub-tile is dead once G is complete
 #pragma unroll
                 for (int hh = 0; hh < 2; ++hh) {
                     if (32 * hh <= rmax) {
@@ -258,16 +267,21 @@ gdn_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                                     pk[e] = pack_bf16((i0 <= r) ? y[8 * ch + 2 * e] : 0.f,
                                                       (i0 + 1 <= r) ? y[8 * ch + 2 * e + 1] : 0.f);
                                 }
-                                st_global_v4(pimg + swz(r, 4 * hh + ch), pk[0], pk[1], pk[2], pk[3]);
+                                st_shared_v4(pimg + swz(r, 4 * hh + ch), pk[0], pk[1], pk[2], pk[3]);
                             }
                         }
                     } else if (!is_a) {
 #pragma unroll
-                        for (int ch = 0; ch < 4; ++ch) st_global_v4(pimg + swz(r, 4 * hh + ch), 0u, 0u, 0u, 0u);
+                        for (int ch = 0; ch < 4; ++ch) st_shared_v4(pimg + swz(r, 4 * hh + ch), 0u, 0u, 0u, 0u);
                     }
                 }
             }
+            fence_proxy_async_smem();
             named_bar_sync(1, 128);
+            // The images leave the SM as bulk copies from shared memory (a thread-per-row store would
+            // touch 32 different lines per instruction); thread 0 issues them and later waits for their
+            // shared-memory reads before the staging space is reused.
+            if (tp == 0) { bulk_store(out_item + IT_P, base + PS_KQ + 8192, 8192); bulk_commit(); }
             // ---- step b2: T = (I + A)^{-1}, blocked forward substitution (fp32) ----
             if (tp < 64) {   // level 0: four 16x16 diagonal blocks, one column per thread
                 const int I = tp >> 4, cc = tp & 15;
@@ -386,12 +400,14 @@ gdn_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                         p2[e] = pack_bf16(t0 * b, t1 * b);
                     }
                     st_shared_v4(base + PS_T1 + swz(cc, 4 * half + ch), p1[0], p1[1], p1[2], p1[3]);
-                    st_global_v4(out_item + IT_T2 + swz(cc, 4 * half + ch), p2[0], p2[1], p2[2], p2[3]);
+                    st_shared_v4(base + PS_A + 8192 + swz(cc, 4 * half + ch), p2[0], p2[1], p2[2], p2[3]);
                 }
             }
             fence_proxy_async_smem();
             tc_fence_before_sync();
             mbar_arrive(w.bar(PB_TREADY));
+            named_bar_sync(1, 128);
+            if (tp == 0) { bulk_store(out_item + IT_T2, base + PS_A + 8192, 8192); bulk_commit(); }
             // ---- step b3 result: -W^T image to scratch; gate vectors to scratch ----
             if (tp < GATE_FLOATS / 4)
                 *reinterpret_cast<float4*>(out_item + IT_GATES + tp * 16) = *reinterpret_cast<const float4*>(gates + 4 * tp);
@@ -408,8 +424,16 @@ gdn_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
 #pragma unroll
                     for (int e = 0; e < 4; ++e)
                         pk[e] = pack_bf16(-__uint_as_float(x[8 * ch + 2 * e]), -__uint_as_float(x[8 * ch + 2 * e + 1]));
-                    st_global_v4(out_item + IT_W + swz(tp, 4 * hh + ch), pk[0], pk[1], pk[2], pk[3]);
+                    st_shared_v4(base + PS_KQ + (tp >> 6) * 16384 + swz(tp & 63, 4 * hh + ch), pk[0], pk[1], pk[2], pk[3]);
                 }
+            }
+            fence_proxy_async_smem();
+            named_bar_sync(1, 128);
+            if (tp == 0) {                                     // rows 0..63 sit over K_lo, rows 64..127 over K_hi
+                bulk_store(out_item + IT_W, base + PS_KQ, 8192);
+                bulk_store(out_item + IT_W + 8192, base + PS_KQ + 16384, 8192);
+                bulk_commit();
+                bulk_wait_read_all();                          // P, T2, W staging may now be overwritten
             }
             tc_fence_before_sync();
             mbar_arrive(w.bar(PB_DONE));
@@ -464,6 +488,7 @@ gdn_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         }
         ++it;
     }
+    if (tid == 0) bulk_wait_all();
     tc_fence_before_sync();
     __syncthreads();
     if (warp == 0) {
