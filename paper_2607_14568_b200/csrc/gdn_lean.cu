@@ -304,82 +304,90 @@ gdn_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                 }
             }
             named_bar_sync(1, 128);
-            {   // level 1: 16-blocks (1,0) and (3,2):  T21 = -T22 (A21 T11)
-                const int pr = tp >> 6, r = (tp >> 2) & 15, cg = tp & 3;
+            // The merges are small fp32 products out of shared memory.  A warp owns 8 rows and a lane one
+            // column: the row operand is read with warp-uniform 16-byte loads (one wavefront each) and
+            // the column operand with one 4-byte load per lane -- shared-memory wavefronts, not FMAs,
+            // bound this kernel.
+            {   // level 1: 16-blocks (1,0) and (3,2):  T21 = -T22 (A21 T11); lanes 16..31 take the second half of i
+                const int pr = warp >> 1, r0 = 8 * (warp & 1), c = lane & 15, ih = lane >> 4;
                 const int lo = 32 * pr, hi = lo + 16;
-                float acc[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll 2
-                for (int i4 = 0; i4 < 4; ++i4) {
-                    const float4 a4 = *reinterpret_cast<const float4*>(sA + (hi + r) * LDA + lo + 4 * i4);
-                    const float av[4] = {a4.x, a4.y, a4.z, a4.w};
+                float acc[8];
 #pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        const float4 t4 = *reinterpret_cast<const float4*>(sTf + (lo + 4 * i4 + e) * LDA + lo + 4 * cg);
-                        acc[0] = fmaf(av[e], t4.x, acc[0]); acc[1] = fmaf(av[e], t4.y, acc[1]);
-                        acc[2] = fmaf(av[e], t4.z, acc[2]); acc[3] = fmaf(av[e], t4.w, acc[3]);
+                for (int x = 0; x < 8; ++x) acc[x] = 0.f;
+#pragma unroll
+                for (int i4 = 0; i4 < 2; ++i4) {
+                    const int ib = 8 * ih + 4 * i4;
+                    float tv[4];
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) tv[e] = sTf[(lo + ib + e) * LDA + lo + c];
+#pragma unroll
+                    for (int x = 0; x < 8; ++x) {
+                        const float4 a4 = *reinterpret_cast<const float4*>(sA + (hi + r0 + x) * LDA + lo + ib);
+                        acc[x] = fmaf(a4.x, tv[0], fmaf(a4.y, tv[1], fmaf(a4.z, tv[2], fmaf(a4.w, tv[3], acc[x]))));
                     }
                 }
-                *reinterpret_cast<float4*>(sY + (16 * pr + r) * LDY + 4 * cg) = make_float4(acc[0], acc[1], acc[2], acc[3]);
+#pragma unroll
+                for (int x = 0; x < 8; ++x) {
+                    acc[x] += __shfl_xor_sync(0xffffffffu, acc[x], 16);
+                    if (ih == 0) sY[(16 * pr + r0 + x) * LDY + c] = acc[x];
+                }
                 named_bar_sync(1, 128);
-                float t[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll 2
-                for (int i4 = 0; i4 < 4; ++i4) {
-                    const float4 a4 = *reinterpret_cast<const float4*>(sTf + (hi + r) * LDA + hi + 4 * i4);
-                    const float av[4] = {a4.x, a4.y, a4.z, a4.w};
 #pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        const float4 y4 = *reinterpret_cast<const float4*>(sY + (16 * pr + 4 * i4 + e) * LDY + 4 * cg);
-                        t[0] = fmaf(av[e], y4.x, t[0]); t[1] = fmaf(av[e], y4.y, t[1]);
-                        t[2] = fmaf(av[e], y4.z, t[2]); t[3] = fmaf(av[e], y4.w, t[3]);
+                for (int x = 0; x < 8; ++x) acc[x] = 0.f;
+#pragma unroll
+                for (int i4 = 0; i4 < 2; ++i4) {
+                    const int ib = 8 * ih + 4 * i4;
+                    float yv[4];
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) yv[e] = sY[(16 * pr + ib + e) * LDY + c];
+#pragma unroll
+                    for (int x = 0; x < 8; ++x) {
+                        const float4 a4 = *reinterpret_cast<const float4*>(sTf + (hi + r0 + x) * LDA + hi + ib);
+                        acc[x] = fmaf(a4.x, yv[0], fmaf(a4.y, yv[1], fmaf(a4.z, yv[2], fmaf(a4.w, yv[3], acc[x]))));
                     }
                 }
-                *reinterpret_cast<float4*>(sTf + (hi + r) * LDA + lo + 4 * cg) = make_float4(-t[0], -t[1], -t[2], -t[3]);
-                *reinterpret_cast<float4*>(sTf + (lo + r) * LDA + hi + 4 * cg) = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+                for (int x = 0; x < 8; ++x) {
+                    acc[x] += __shfl_xor_sync(0xffffffffu, acc[x], 16);
+                    if (ih == 0) sTf[(hi + r0 + x) * LDA + lo + c] = -acc[x];
+                    else sTf[(lo + r0 + x) * LDA + hi + c] = 0.f;      // the upper-right 16-blocks are zero
+                }
             }
             named_bar_sync(1, 128);
             {   // level 2: the 32-block (1,0)
-                const int r = tp >> 2, cg = tp & 3;
+                const int r0 = 8 * warp, c = lane;
                 float acc[8];
 #pragma unroll
-                for (int e = 0; e < 8; ++e) acc[e] = 0.f;
+                for (int x = 0; x < 8; ++x) acc[x] = 0.f;
 #pragma unroll 2
                 for (int i4 = 0; i4 < 8; ++i4) {
-                    const float4 a4 = *reinterpret_cast<const float4*>(sA + (32 + r) * LDA + 4 * i4);
-                    const float av[4] = {a4.x, a4.y, a4.z, a4.w};
+                    float tv[4];
 #pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        const float* trow = sTf + (4 * i4 + e) * LDA + 8 * cg;
-                        const float4 t0 = *reinterpret_cast<const float4*>(trow);
-                        const float4 t1 = *reinterpret_cast<const float4*>(trow + 4);
-                        acc[0] = fmaf(av[e], t0.x, acc[0]); acc[1] = fmaf(av[e], t0.y, acc[1]);
-                        acc[2] = fmaf(av[e], t0.z, acc[2]); acc[3] = fmaf(av[e], t0.w, acc[3]);
-                        acc[4] = fmaf(av[e], t1.x, acc[4]); acc[5] = fmaf(av[e], t1.y, acc[5]);
-                        acc[6] = fmaf(av[e], t1.z, acc[6]); acc[7] = fmaf(av[e], t1.w, acc[7]);
+                    for (int e = 0; e < 4; ++e) tv[e] = sTf[(4 * i4 + e) * LDA + c];
+#pragma unroll
+                    for (int x = 0; x < 8; ++x) {
+                        const float4 a4 = *reinterpret_cast<const float4*>(sA + (32 + r0 + x) * LDA + 4 * i4);
+                        acc[x] = fmaf(a4.x, tv[0], fmaf(a4.y, tv[1], fmaf(a4.z, tv[2], fmaf(a4.w, tv[3], acc[x]))));
                     }
                 }
-                *reinterpret_cast<float4*>(sY + r * LDY + 8 * cg) = make_float4(acc[0], acc[1], acc[2], acc[3]);
-                *reinterpret_cast<float4*>(sY + r * LDY + 8 * cg + 4) = make_float4(acc[4], acc[5], acc[6], acc[7]);
+#pragma unroll
+                for (int x = 0; x < 8; ++x) sY[(r0 + x) * LDY + c] = acc[x];
                 named_bar_sync(1, 128);
-                float t[8];
 #pragma unroll
-                for (int e = 0; e < 8; ++e) t[e] = 0.f;
+                for (int x = 0; x < 8; ++x) acc[x] = 0.f;
 #pragma unroll 2
                 for (int i4 = 0; i4 < 8; ++i4) {
-                    const float4 a4 = *reinterpret_cast<const float4*>(sTf + (32 + r) * LDA + 32 + 4 * i4);
-                    const float av[4] = {a4.x, a4.y, a4.z, a4.w};
+                    float yv[4];
 #pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        const float* yrow = sY + (4 * i4 + e) * LDY + 8 * cg;
-                        const float4 y0 = *reinterpret_cast<const float4*>(yrow);
-                        const float4 y1 = *reinterpret_cast<const float4*>(yrow + 4);
-                        t[0] = fmaf(av[e], y0.x, t[0]); t[1] = fmaf(av[e], y0.y, t[1]);
-                        t[2] = fmaf(av[e], y0.z, t[2]); t[3] = fmaf(av[e], y0.w, t[3]);
-                        t[4] = fmaf(av[e], y1.x, t[4]); t[5] = fmaf(av[e], y1.y, t[5]);
-                        t[6] = fmaf(av[e], y1.z, t[6]); t[7] = fmaf(av[e], y1.w, t[7]);
+                    for (int e = 0; e < 4; ++e) yv[e] = sY[(4 * i4 + e) * LDY + c];
+#pragma unroll
+                    for (int x = 0; x < 8; ++x) {
+                        const float4 a4 = *reinterpret_cast<const float4*>(sTf + (32 + r0 + x) * LDA + 32 + 4 * i4);
+                        acc[x] = fmaf(a4.x, yv[0], fmaf(a4.y, yv[1], fmaf(a4.z, yv[2], fmaf(a4.w, yv[3], acc[x]))));
                     }
                 }
-                *reinterpret_cast<float4*>(sTf + (32 + r) * LDA + 8 * cg) = make_float4(-t[0], -t[1], -t[2], -t[3]);
-                *reinterpret_cast<float4*>(sTf + (32 + r) * LDA + 8 * cg + 4) = make_float4(-t[4], -t[5], -t[6], -t[7]);
+#pragma unroll
+                for (int x = 0; x < 8; ++x) sTf[(32 + r0 + x) * LDA + c] = -acc[x];
             }
             named_bar_sync(1, 128);
             // ---- step b3 operands: row i = cc of (T diag(b e^g))^T (shared) and (T diag(b))^T (scratch) ----
