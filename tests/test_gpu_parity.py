@@ -129,6 +129,17 @@ def test_two_kernel_sequence_split(T, nseg, gate):
         gdn.lib().gdn_debug_force_segments(0)
 
 
+def test_two_kernel_sequence_split_wide_values_and_batch():
+    """Sequence split with d_v = 256 (two value blocks share one M chain) and B = 2."""
+    cfg = get_config("large", B=2, T=1100, H=2, seed=77)
+    x = make_inputs(cfg)
+    gdn.lib().gdn_debug_force_segments(3)
+    try:
+        check_bf16(x, prefill_two_kernel, "split d_v=256 B=2")
+    finally:
+        gdn.lib().gdn_debug_force_segments(0)
+
+
 def test_bf16_special_cases():
     """beta = 0 gives pure decay of the initial state; identity padding changes nothing."""
     cfg = get_config("long", T=192, H=2, seed=41)
