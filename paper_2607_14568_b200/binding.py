@@ -54,6 +54,10 @@ def lib():
         L.gdn_set_workspace.restype = i
         L.gdn_debug_force_path.argtypes = [i]
         L.gdn_debug_force_path.restype = None
+        L.gdn_debug_drop_chunk.argtypes = [i]
+        L.gdn_debug_drop_chunk.restype = None
+        L.gdn_debug_reset_status.argtypes = []
+        L.gdn_debug_reset_status.restype = i
         L.gdn_debug_set_timing.argtypes = [i]
         L.gdn_debug_set_timing.restype = i
         L.gdn_debug_get_timing.argtypes = [ctypes.POINTER(ctypes.c_float)]

@@ -198,6 +198,12 @@ int gdn_query_status(void) { return tc_query_status(); }
 // Not part of the public header: 0 = automatic, 1 = fused kernel only, 2 = two-kernel pipeline only.
 void gdn_debug_force_path(int path) { g_force_path = path; }
 
+// Not part of the public header: failure-path test hooks.  gdn_debug_drop_chunk(c) makes the chain
+// kernel's TMA thread of one CTA skip chunk c, so the bounded waits on that data expire;
+// gdn_debug_reset_status() clears the status word afterwards.
+void gdn_debug_drop_chunk(int chunk) { lean_set_drop_chunk(chunk); }
+int gdn_debug_reset_status(void) { return lean_reset_status(); }
+
 // Not part of the public header: per-kernel event timing of the two-kernel pipeline (benchmark).
 int gdn_debug_set_timing(int enable) { return lean_set_timing(enable); }
 int gdn_debug_get_timing(float* ms4) { return ms4 ? lean_get_timing(ms4) : GDN_ERR_INVALID_ARG; }

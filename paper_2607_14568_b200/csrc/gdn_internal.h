@@ -45,6 +45,8 @@ int launch_lean(const PrefillArgs& a, void* workspace, size_t workspace_bytes, c
 int launch_lean_static(const PrefillArgs& a, cudaStream_t stream);   // built-in scratch, allocates nothing
 int lean_query_status();
 void lean_force_segments(int nseg);   // tests only: 0 = automatic plan
+void lean_set_drop_chunk(int c);      // tests only: make one TMA load never happen (bounded waits expire)
+int lean_reset_status();              // tests only: clear the status word
 void lean_set_debug(float* p);        // tests only: time stamps of the chain kernel
 int lean_set_timing(int enable);      // benchmark only: record events around each kernel
 int lean_get_timing(float* ms4);      // {prepare, summary, combine, chain} of the last call

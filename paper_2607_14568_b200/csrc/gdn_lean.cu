@@ -38,6 +38,7 @@ static bool g_lean_timing = false;
 static cudaEvent_t g_lean_events[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};
 static bool g_lean_split_last = false;
 static float* g_lean_dbg = nullptr;        // debug: time stamps of the chain kernel
+static int g_lean_drop_chunk = -1;         // tests: chunk the chain kernel's TMA thread skips (-1 = none)
 
 namespace {
 
@@ -541,6 +542,8 @@ struct ChainParams {
     const uint8_t* items;
     const float* seg_sin;     // [B*nseg, H, d_k, d_v] incoming states of segments 1.. (sequence split), or nullptr
     float* dbg;               // debug build: time stamps of CTA (0,0,0), [role][chunk < 32][event < 8], ns
+    int drop_chunk;           // tests only: the TMA thread of CTA (0,0,0) never loads this chunk (-1 = off), so
+                              // that the bounded waits on it expire and the abort path runs
     int B, T, H, dv;
     int nseg, seg_chunks;     // segments per sequence (1 = no split) and chunks per segment
 };
@@ -798,6 +801,7 @@ gdn_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             prefetch_tensormap(&map_k);
             prefetch_tensormap(&map_v);
             for (int c = 0; c < nchunks; ++c) {
+                if (c == p.drop_chunk && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0) continue;
                 const int tok = (int)(tok0 + (long)c * C);
                 const uint8_t* item = p.items + (size_t)((slot0 + c) * H + h) * ITEM_BYTES;
                 {   // ring B: V tile and (T diag(b))^T
@@ -1275,7 +1279,7 @@ int launch_lean(const PrefillArgs& a, void* workspace, size_t workspace_bytes, c
     g_lean_split_last = nseg > 1;
     // ---- steps c, d ----
     ChainParams cp{a.initial_state, static_cast<__nv_bfloat16*>(a.out), a.final_state, a.cu_seqlens,
-                   ws, seg_sin, g_lean_dbg, a.B, a.T, a.H, a.d_v, nseg, seg_chunks};
+                   ws, seg_sin, g_lean_dbg, g_lean_drop_chunk, a.B, a.T, a.H, a.d_v, nseg, seg_chunks};
     dim3 grid(a.d_v / DVB, a.H, a.B * nseg);
     if (g_lean_dbg) gdn_chain_kernel<true><<<grid, CHAIN_THREADS, CHAIN_SMEM, stream>>>(mq, mk, mv, cp);
     else gdn_chain_kernel<false><<<grid, CHAIN_THREADS, CHAIN_SMEM, stream>>>(mq, mk, mv, cp);
@@ -1286,6 +1290,11 @@ int launch_lean(const PrefillArgs& a, void* workspace, size_t workspace_bytes, c
 
 void lean_force_segments(int nseg) { g_lean_force_nseg = nseg; }
 void lean_set_debug(float* p) { g_lean_dbg = p; }
+void lean_set_drop_chunk(int c) { g_lean_drop_chunk = c; }
+int lean_reset_status() {
+    const int zero = 0;
+    return cudaMemcpyToSymbol(g_lean_status, &zero, sizeof(int)) == cudaSuccess ? GDN_OK : GDN_ERR_CUDA;
+}
 
 int lean_set_timing(int enable) {
     if (enable)
@@ -1371,7 +1380,7 @@ int launch_lean_static(const PrefillArgs& a, cudaStream_t stream) {
     if (cudaGetLastError() != cudaSuccess) return GDN_ERR_CUDA;
     const int nch = packed ? 1 : (a.T + C - 1) / C;            // one segment: the whole sequence
     ChainParams cp{a.initial_state, static_cast<__nv_bfloat16*>(a.out), a.final_state, a.cu_seqlens,
-                   ws, nullptr, nullptr, a.B, a.T, a.H, a.d_v, 1, packed ? (1 << 24) : (nch > 0 ? nch : 1)};
+                   ws, nullptr, nullptr, -1, a.B, a.T, a.H, a.d_v, 1, packed ? (1 << 24) : (nch > 0 ? nch : 1)};
     dim3 grid(a.d_v / DVB, a.H, a.B);
     gdn_chain_kernel<false><<<grid, CHAIN_THREADS, CHAIN_SMEM, stream>>>(mq, mk, mv, cp);
     count_launch();
