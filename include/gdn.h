@@ -141,6 +141,24 @@ int gdn_decode_step(const void* q, const void* k, const void* v,
                     gdn_stream_t stream);
 
 /*
+ * gdn_chunk_prefill that also returns the recurrent state at chunk boundaries: the material of a
+ * position-indexed prefix-snapshot cache (Section "An All-GPU Engine for the Hybrid Backbone": the
+ * serving process keeps snapshots of the recurrent state by position).  Batched input only (no
+ * cu_seqlens).  snapshots is [B, n_snap, H, d_k, d_v] fp32 with n_snap = (T / 64) /
+ * snapshot_every_chunks; entry i holds the state after token (i + 1) * snapshot_every_chunks * 64
+ * of each sequence -- exactly what initial_state must be to resume the prefill there.  Needs the
+ * scratch of gdn_set_workspace (GDN_ERR_WORKSPACE without it); other arguments, support and
+ * errors as gdn_chunk_prefill with d_k = 128, d_v a multiple of 128.
+ */
+int gdn_chunk_prefill_snapshots(const void* q, const void* k, const void* v,
+                                const float* log_alpha, const float* beta,
+                                const float* initial_state,
+                                void* out, float* final_state,
+                                int B, int T, int H, int d_k, int d_v, int chunk,
+                                int snapshot_every_chunks, float* snapshots,
+                                gdn_stream_t stream);
+
+/*
  * Optional scratch memory.  Without it gdn_chunk_prefill runs one fused kernel per call in
  * which each (sequence, head) chain also does its own forward substitutions.  With scratch of
  * at least gdn_workspace_bytes(...) bytes the state-independent steps (cumulative gate,

@@ -48,6 +48,8 @@ def lib():
         L.gdn_host_staging_bytes.restype = sz
         L.gdn_decode_step.argtypes = [vp] * 7 + [i] * 4 + [vp]
         L.gdn_decode_step.restype = i
+        L.gdn_chunk_prefill_snapshots.argtypes = [vp] * 8 + [i] * 7 + [vp, vp]
+        L.gdn_chunk_prefill_snapshots.restype = i
         L.gdn_workspace_bytes.argtypes = [i] * 6
         L.gdn_workspace_bytes.restype = sz
         L.gdn_set_workspace.argtypes = [vp, sz]
@@ -197,6 +199,28 @@ def gdn_chunk_prefill_noalloc(q, k, v, log_alpha, beta, initial_state, out, fina
     does not fit.  Make the first call on a device outside stream capture; do not overlap calls."""
     return _prefill("gdn_chunk_prefill_noalloc", torch.bfloat16, q, k, v, log_alpha, beta, initial_state,
                     out, final_state, cu_seqlens, chunk, stream)
+
+
+def gdn_chunk_prefill_snapshots(q, k, v, log_alpha, beta, initial_state, out, final_state, snapshot_every_chunks,
+                                snapshots, chunk: int = 64, stream=None):
+    """gdn_chunk_prefill (batched input) that also writes the state after every ``snapshot_every_chunks``
+    chunks into ``snapshots`` [B, n_snap, H, d_k, d_v] fp32.  Needs gdn_set_workspace.  See include/gdn.h."""
+    f32, bf = torch.float32, torch.bfloat16
+    _check([("q", q, bf), ("k", k, bf), ("v", v, bf), ("out", out, bf), ("log_alpha", log_alpha, f32),
+            ("beta", beta, f32), ("initial_state", initial_state, f32), ("final_state", final_state, f32),
+            ("snapshots", snapshots, f32)], bf, "cuda")
+    B, T, H, d_k = q.shape
+    d_v = v.shape[-1]
+    n_snap = (T // 64) // int(snapshot_every_chunks)
+    if tuple(snapshots.shape) != (B, n_snap, H, d_k, d_v):
+        raise ValueError("snapshots must be [B, (T//64)//every, H, d_k, d_v]")
+    rc = lib().gdn_chunk_prefill_snapshots(_ptr(q), _ptr(k), _ptr(v), _ptr(log_alpha), _ptr(beta),
+                                           _ptr(initial_state), _ptr(out), _ptr(final_state), int(B), int(T), int(H),
+                                           int(d_k), int(d_v), int(chunk), int(snapshot_every_chunks),
+                                           _ptr(snapshots), _stream(stream))
+    if rc != 0:
+        raise GdnError(rc, "gdn_chunk_prefill_snapshots")
+    return out, final_state, snapshots
 
 
 def gdn_decode_step(q, k, v, log_alpha, beta, state, out, stream=None):

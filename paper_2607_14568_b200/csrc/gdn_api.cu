@@ -182,6 +182,23 @@ int gdn_decode_step(const void* q, const void* k, const void* v, const float* lo
     return launch_decode(q, k, v, log_alpha, beta, state, out, B, H, d_k, d_v, reinterpret_cast<cudaStream_t>(stream));
 }
 
+int gdn_chunk_prefill_snapshots(const void* q, const void* k, const void* v, const float* log_alpha,
+                                const float* beta, const float* initial_state, void* out, float* final_state,
+                                int B, int T, int H, int d_k, int d_v, int chunk,
+                                int snapshot_every_chunks, float* snapshots, gdn_stream_t stream) {
+    const PrefillArgs a = pack(q, k, v, log_alpha, beta, initial_state, out, final_state, nullptr, B, T, H, d_k, d_v);
+    if (int rc = validate(a, chunk)) return rc;
+    if (snapshot_every_chunks <= 0) return GDN_ERR_INVALID_ARG;
+    if ((T / kChunk) / snapshot_every_chunks == 0) snapshots = nullptr;   // no boundary reached: nothing to write
+    else if (!snapshots) return GDN_ERR_INVALID_ARG;
+    if (!aligned16(snapshots) || !tc_supported(d_k, d_v)) return GDN_ERR_UNSUPPORTED;
+    if (T == 0) return launch_tc(a, reinterpret_cast<cudaStream_t>(stream));
+    const size_t need = lean_workspace_bytes(B, T, H, d_k, d_v, false);
+    if (!g_workspace || g_workspace_bytes < need) return GDN_ERR_WORKSPACE;
+    return launch_lean(a, g_workspace, g_workspace_bytes, reinterpret_cast<cudaStream_t>(stream), snapshots,
+                       snapshot_every_chunks);
+}
+
 size_t gdn_workspace_bytes(int B, int T, int H, int d_k, int d_v, int packed) {
     return lean_workspace_bytes(B, T, H, d_k, d_v, packed != 0);
 }

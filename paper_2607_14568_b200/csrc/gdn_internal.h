@@ -41,7 +41,9 @@ bool tc_make_map(CUtensorMap* map, const void* ptr, uint64_t tokens, uint64_t H,
 
 // Two-kernel pipeline (prepare on all SMs, then the chain) using caller-provided scratch.
 size_t lean_workspace_bytes(int B, int T, int H, int d_k, int d_v, bool packed);
-int launch_lean(const PrefillArgs& a, void* workspace, size_t workspace_bytes, cudaStream_t stream);
+// snaps (optional, batched input only): [B, (T/64)/snap_every, H, d_k, d_v], the state after every snap_every chunks
+int launch_lean(const PrefillArgs& a, void* workspace, size_t workspace_bytes, cudaStream_t stream,
+                float* snaps = nullptr, int snap_every = 1);
 int launch_lean_static(const PrefillArgs& a, cudaStream_t stream);   // built-in scratch, allocates nothing
 int lean_query_status();
 void lean_force_segments(int nseg);   // tests only: 0 = automatic plan

@@ -546,6 +546,8 @@ struct ChainParams {
                               // that the bounded waits on it expire and the abort path runs
     int B, T, H, dv;
     int nseg, seg_chunks;     // segments per sequence (1 = no split) and chunks per segment
+    float* snaps;             // optional [B, nsnap, H, d_k, d_v]: the state after every snap_every chunks
+    int snap_every, nsnap;
 };
 
 template <bool DBG>
@@ -686,6 +688,15 @@ gdn_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             tc_fence_before_sync();
             mbar_arrive(w.bar(CB_SREADY));
             if (tid == 0) stamp(0, c, 3);
+            if (p.snaps) {                              // state snapshot at a chunk boundary (off the chain: plain stores)
+                const int gc = cbeg + c + 1;            // chunks of the sequence consumed so far
+                if (gc % p.snap_every == 0 && gc / p.snap_every <= p.nsnap && gc * C <= sq.len) {
+                    float* dst = p.snaps + (((size_t)n * p.nsnap + (gc / p.snap_every - 1)) * H + h) * DK * dv +
+                                 (size_t)dvb * DVB + j;
+#pragma unroll
+                    for (int m = 0; m < DK; ++m) dst[(size_t)m * dv] = S[m];
+                }
+            }
         }
         if (p.sT && seg == p.nseg - 1) {
 #pragma unroll
@@ -1210,7 +1221,8 @@ size_t lean_workspace_bytes(int B, int T, int H, int d_k, int d_v, bool packed) 
     return bytes;
 }
 
-int launch_lean(const PrefillArgs& a, void* workspace, size_t workspace_bytes, cudaStream_t stream) {
+int launch_lean(const PrefillArgs& a, void* workspace, size_t workspace_bytes, cudaStream_t stream,
+                float* snaps, int snap_every) {
     if (!tc_supported(a.d_k, a.d_v)) return GDN_ERR_UNSUPPORTED;
     if (a.H > 65535 || a.B > 4095) return GDN_ERR_UNSUPPORTED;
     const bool packed = a.cu_seqlens != nullptr;
@@ -1279,7 +1291,8 @@ int launch_lean(const PrefillArgs& a, void* workspace, size_t workspace_bytes, c
     g_lean_split_last = nseg > 1;
     // ---- steps c, d ----
     ChainParams cp{a.initial_state, static_cast<__nv_bfloat16*>(a.out), a.final_state, a.cu_seqlens,
-                   ws, seg_sin, g_lean_dbg, g_lean_drop_chunk, a.B, a.T, a.H, a.d_v, nseg, seg_chunks};
+                   ws, seg_sin, g_lean_dbg, g_lean_drop_chunk, a.B, a.T, a.H, a.d_v, nseg, seg_chunks,
+                   snaps, snap_every, snaps ? (a.T / C) / snap_every : 0};
     dim3 grid(a.d_v / DVB, a.H, a.B * nseg);
     if (g_lean_dbg) gdn_chain_kernel<true><<<grid, CHAIN_THREADS, CHAIN_SMEM, stream>>>(mq, mk, mv, cp);
     else gdn_chain_kernel<false><<<grid, CHAIN_THREADS, CHAIN_SMEM, stream>>>(mq, mk, mv, cp);
@@ -1380,7 +1393,8 @@ int launch_lean_static(const PrefillArgs& a, cudaStream_t stream) {
     if (cudaGetLastError() != cudaSuccess) return GDN_ERR_CUDA;
     const int nch = packed ? 1 : (a.T + C - 1) / C;            // one segment: the whole sequence
     ChainParams cp{a.initial_state, static_cast<__nv_bfloat16*>(a.out), a.final_state, a.cu_seqlens,
-                   ws, nullptr, nullptr, -1, a.B, a.T, a.H, a.d_v, 1, packed ? (1 << 24) : (nch > 0 ? nch : 1)};
+                   ws, nullptr, nullptr, -1, a.B, a.T, a.H, a.d_v, 1, packed ? (1 << 24) : (nch > 0 ? nch : 1),
+                   nullptr, 1, 0};
     dim3 grid(a.d_v / DVB, a.H, a.B);
     gdn_chain_kernel<false><<<grid, CHAIN_THREADS, CHAIN_SMEM, stream>>>(mq, mk, mv, cp);
     count_launch();
