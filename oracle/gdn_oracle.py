@@ -11,6 +11,11 @@ the C file: ``q,k [B,T,H,d_k]``, ``v [B,T,H,d_v]``, ``log_alpha,beta [B,T,H]``,
   chunked     the intra-/inter-chunk form of the same section (form=1: its
               S' = M S + N variant)
   dense       the whole sequence as one general linear system (brute force)
+  prologue    the per-position kernels in front of the scan (Section "Batched prefill":
+              norms and gating batched over the chunk): L2 norm of q and k over the feature
+              axis, beta = sigmoid(b), log_alpha = -softplus(a) * gate_scale.  The paper names
+              these kernels without printing formulas; the forms here are the reading the
+              benchmark inputs were drawn with.  Plain numpy, fp64.
 """
 from __future__ import annotations
 
@@ -104,3 +109,14 @@ def chunked(q, k, v, log_alpha, beta, initial_state=None, cu_seqlens=None, chunk
 def dense(q, k, v, log_alpha, beta, initial_state=None, cu_seqlens=None):
     arrs, dims = _prepare(q, k, v, log_alpha, beta, initial_state, cu_seqlens)
     return _call(_load().gdn_oracle_dense, arrs, dims)
+
+
+def prologue(q_raw, k_raw, a_raw, b_raw, gate_scale, eps=0.0):
+    """(q, k, log_alpha, beta) in fp64 from raw projections:
+    x / sqrt(sum_f x_f^2 + eps) per (token, head) for q and k, 1 / (1 + e^{-b}), -ln(1 + e^{a}) * gate_scale."""
+    q_raw, k_raw, a_raw, b_raw = _f64(q_raw), _f64(k_raw), _f64(a_raw), _f64(b_raw)
+    q = q_raw / np.sqrt((q_raw * q_raw).sum(axis=-1, keepdims=True) + float(eps))
+    k = k_raw / np.sqrt((k_raw * k_raw).sum(axis=-1, keepdims=True) + float(eps))
+    beta = 1.0 / (1.0 + np.exp(-b_raw))
+    log_alpha = -np.log(1.0 + np.exp(a_raw)) * float(gate_scale)
+    return q, k, log_alpha, beta

@@ -220,3 +220,49 @@ def test_oracle_rejects_bad_arguments():
         oracle.sequential(q[0], k[0], v[0], la[0], beta[0], None, cu_seqlens=np.array([0, 3], dtype=np.int32))
     with pytest.raises(ValueError):
         oracle.chunked(q, k, v, la, beta, None, chunk=0)
+
+
+# ---------------------------------------------------------------------------
+# prologue (norms and gating in front of the scan)
+# ---------------------------------------------------------------------------
+def test_prologue_closed_forms():
+    # 3-4-5 triangle: the unit vector of (3, 4) is (0.6, 0.8); of (0, -2) it is (0, -1)
+    q_raw = np.array([[[3.0, 4.0]], [[0.0, -2.0]]])            # [T=2, H=1, d=2]
+    k_raw = np.array([[[5.0, 12.0]], [[-8.0, 6.0]]])           # 5-12-13 and 6-8-10
+    a_raw = np.array([[0.0], [np.log(np.e - 1.0)]])            # softplus = ln 2 and exactly 1
+    b_raw = np.array([[0.0], [np.log(3.0)]])                   # sigmoid = 1/2 and 3/4
+    q, k, la, be = oracle.prologue(q_raw, k_raw, a_raw, b_raw, gate_scale=0.25)
+    np.testing.assert_allclose(q, [[[0.6, 0.8]], [[0.0, -1.0]]], rtol=1e-15, atol=0)
+    np.testing.assert_allclose(k, [[[5 / 13, 12 / 13]], [[-0.8, 0.6]]], rtol=1e-15, atol=0)
+    np.testing.assert_allclose(la, [[-0.25 * np.log(2.0)], [-0.25]], rtol=1e-15)
+    np.testing.assert_allclose(be, [[0.5], [0.75]], rtol=1e-15)
+    # eps enters under the square root: (3,4) with eps = 11 has length 6
+    q2, *_ = oracle.prologue(q_raw, k_raw, a_raw, b_raw, gate_scale=1.0, eps=11.0)
+    np.testing.assert_allclose(q2[0, 0], [0.5, 4.0 / 6.0], rtol=1e-15)
+
+
+def test_prologue_invariants():
+    rng = np.random.default_rng(21)
+    q_raw = rng.standard_normal((2, 9, 3, 16)) * np.exp(rng.standard_normal((2, 9, 3, 1)))
+    k_raw = rng.standard_normal((2, 9, 3, 16)) * 7.0
+    a_raw = rng.standard_normal((2, 9, 3)) * 3
+    b_raw = rng.standard_normal((2, 9, 3)) * 3
+    q, k, la, be = oracle.prologue(q_raw, k_raw, a_raw, b_raw, gate_scale=0.05)
+    np.testing.assert_allclose(np.linalg.norm(q, axis=-1), 1.0, rtol=1e-14)
+    np.testing.assert_allclose(np.linalg.norm(k, axis=-1), 1.0, rtol=1e-14)
+    # direction kept (cosine with the raw vector is +1), positive rescaling changes nothing
+    assert ((q * q_raw).sum(-1) > 0).all()
+    q3, k3, _, _ = oracle.prologue(q_raw * 3.5, k_raw * 0.01, a_raw, b_raw, gate_scale=0.05)
+    np.testing.assert_allclose(q3, q, rtol=1e-13)
+    np.testing.assert_allclose(k3, k, rtol=1e-13)
+    # sigmoid(x) + sigmoid(-x) = 1; softplus(x) - softplus(-x) = x; gate in (0, 1]; linear in the scale
+    _, _, la_neg, be_neg = oracle.prologue(q_raw, k_raw, -a_raw, -b_raw, gate_scale=0.05)
+    np.testing.assert_allclose(be + be_neg, 1.0, rtol=1e-14)
+    np.testing.assert_allclose((la_neg - la) / 0.05, a_raw, rtol=1e-12, atol=1e-13)
+    assert (la < 0).all() and ((be > 0) & (be < 1)).all()
+    _, _, la2, _ = oracle.prologue(q_raw, k_raw, a_raw, b_raw, gate_scale=0.1)
+    np.testing.assert_allclose(la2, 2 * la, rtol=1e-15)
+    # agrees with scipy's independently written special functions
+    from scipy.special import expit, log1p, logsumexp  # noqa: F401
+    np.testing.assert_allclose(be, expit(b_raw), rtol=1e-14)
+    np.testing.assert_allclose(la, -0.05 * np.logaddexp(0.0, a_raw), rtol=1e-13)

@@ -17,6 +17,10 @@ Distributions (per token and head):
   beta       sigmoid(N(0,1))                      fp32
   log_alpha  -softplus(N(0,1)) * gate_scale       fp32 (natural log of the gate)
   S0         N(0, init_std) fp32, or absent (zeros) when init_std == 0
+With ``raw=True`` the tensors are the raw projections instead, for the entry point that
+runs the norms and gating itself: q, k are N(0,1) times a per-(token, head) magnitude
+exp(N(0, 0.5)) and are not normalised, and the ``beta`` / ``log_alpha`` fields hold the N(0,1)
+pre-activations (the call is given ``gate_scale``).
 q, k, v are then rounded to the storage type (bf16 round-to-nearest-even, or kept
 fp32).  bf16 tensors are returned as uint16 bit patterns.
 """
@@ -44,6 +48,7 @@ class GdnConfig:
     chunk: int = 64
     varlen: Optional[Tuple[int, int]] = None   # (lo, hi): packed sequences, lengths ~ U{lo..hi}
     lengths: Optional[Tuple[int, ...]] = None  # explicit packed lengths (overrides varlen)
+    raw: bool = False           # raw projections: q, k not normalised, gates left as pre-activations
 
     @property
     def packed(self) -> bool:
@@ -119,13 +124,19 @@ def chain_inputs(cfg: GdnConfig, n: int, h: int, length: Optional[int] = None) -
     v = rng.standard_normal((L, cfg.d_v), dtype=np.float32)
     braw = rng.standard_normal(L, dtype=np.float32)
     araw = rng.standard_normal(L, dtype=np.float32)
-    q /= np.linalg.norm(q, axis=-1, keepdims=True)
-    k /= np.linalg.norm(k, axis=-1, keepdims=True)
-    beta = (1.0 / (1.0 + np.exp(-braw.astype(np.float64)))).astype(np.float32)
-    log_alpha = (-np.logaddexp(0.0, araw.astype(np.float64)) * cfg.gate_scale).astype(np.float32)
+    if not cfg.raw:
+        q /= np.linalg.norm(q, axis=-1, keepdims=True)
+        k /= np.linalg.norm(k, axis=-1, keepdims=True)
+        beta = (1.0 / (1.0 + np.exp(-braw.astype(np.float64)))).astype(np.float32)
+        log_alpha = (-np.logaddexp(0.0, araw.astype(np.float64)) * cfg.gate_scale).astype(np.float32)
+    else:
+        beta, log_alpha = braw, araw
     s0 = None
     if cfg.init_std > 0.0:
         s0 = (rng.standard_normal((cfg.d_k, cfg.d_v), dtype=np.float32) * np.float32(cfg.init_std))
+    if cfg.raw:     # drawn last, so that every other tensor is the same as without raw
+        q *= np.exp(0.5 * rng.standard_normal((L, 1), dtype=np.float32))
+        k *= np.exp(0.5 * rng.standard_normal((L, 1), dtype=np.float32))
     return {"q": _store(q, cfg.dtype), "k": _store(k, cfg.dtype), "v": _store(v, cfg.dtype),
             "beta": beta, "log_alpha": log_alpha, "s0": s0}
 
