@@ -159,6 +159,30 @@ int gdn_chunk_prefill_snapshots(const void* q, const void* k, const void* v,
                                 gdn_stream_t stream);
 
 /*
+ * gdn_chunk_prefill with the per-position prologue fused in (Section "Batched prefill": the norms
+ * and gating around the projections are batched over the chunk).  q_raw, k_raw are the raw bf16
+ * projections and a_raw, b_raw the fp32 gate pre-activations, same shapes as q, k, log_alpha, beta
+ * of gdn_chunk_prefill.  The call computes, per (token, head),
+ *   q = q_raw / sqrt(sum_f q_raw_f^2 + norm_eps)      k likewise
+ *   beta = 1 / (1 + e^{-b_raw})                        log_alpha = -ln(1 + e^{a_raw}) * gate_scale
+ * and then the prefill of gdn_chunk_prefill on them; the normalised q, k are never written to
+ * memory (the inverse norms are folded into the masks and gate vectors in fp32, so they see the
+ * unrounded norm).  The paper names these kernels without printing formulas; these are the forms
+ * the benchmark inputs are drawn with.  A row whose sum of squares plus norm_eps is zero counts
+ * as a zero vector.  gate_scale >= 0, norm_eps >= 0 (else GDN_ERR_INVALID_ARG).  Needs the
+ * scratch of gdn_set_workspace (GDN_ERR_WORKSPACE without it); other arguments, support and
+ * errors as gdn_chunk_prefill with d_k = 128, d_v a multiple of 128.
+ */
+int gdn_chunk_prefill_raw(const void* q_raw, const void* k_raw, const void* v,
+                          const float* a_raw, const float* b_raw,
+                          float gate_scale, float norm_eps,
+                          const float* initial_state,
+                          void* out, float* final_state,
+                          const int32_t* cu_seqlens,
+                          int B, int T, int H, int d_k, int d_v, int chunk,
+                          gdn_stream_t stream);
+
+/*
  * Optional scratch memory.  Without it gdn_chunk_prefill runs one fused kernel per call in
  * which each (sequence, head) chain also does its own forward substitutions.  With scratch of
  * at least gdn_workspace_bytes(...) bytes the state-independent steps (cumulative gate,

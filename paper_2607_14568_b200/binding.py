@@ -50,6 +50,8 @@ def lib():
         L.gdn_decode_step.restype = i
         L.gdn_chunk_prefill_snapshots.argtypes = [vp] * 8 + [i] * 7 + [vp, vp]
         L.gdn_chunk_prefill_snapshots.restype = i
+        L.gdn_chunk_prefill_raw.argtypes = [vp] * 5 + [ctypes.c_float] * 2 + [vp] * 4 + [i] * 6 + [vp]
+        L.gdn_chunk_prefill_raw.restype = i
         L.gdn_workspace_bytes.argtypes = [i] * 6
         L.gdn_workspace_bytes.restype = sz
         L.gdn_set_workspace.argtypes = [vp, sz]
@@ -221,6 +223,30 @@ def gdn_chunk_prefill_snapshots(q, k, v, log_alpha, beta, initial_state, out, fi
     if rc != 0:
         raise GdnError(rc, "gdn_chunk_prefill_snapshots")
     return out, final_state, snapshots
+
+
+def gdn_chunk_prefill_raw(q_raw, k_raw, v, a_raw, b_raw, gate_scale, norm_eps, initial_state, out, final_state,
+                          cu_seqlens=None, chunk: int = 64, stream=None):
+    """gdn_chunk_prefill on raw projections: the L2 norms of q, k and the gates sigmoid(b_raw),
+    -softplus(a_raw) * gate_scale are computed inside the kernels.  Needs gdn_set_workspace.  See include/gdn.h."""
+    f32, bf = torch.float32, torch.bfloat16
+    _check([("q_raw", q_raw, bf), ("k_raw", k_raw, bf), ("v", v, bf), ("out", out, bf), ("a_raw", a_raw, f32),
+            ("b_raw", b_raw, f32), ("initial_state", initial_state, f32), ("final_state", final_state, f32),
+            ("cu_seqlens", cu_seqlens, torch.int32)], bf, "cuda")
+    B, T, H, d_k, d_v = _dims(q_raw, v, cu_seqlens)
+    if k_raw.shape != q_raw.shape or v.shape[:-1] != q_raw.shape[:-1] or out.shape != v.shape:
+        raise ValueError("q, k, v, out shapes disagree")
+    if a_raw.shape != q_raw.shape[:-1] or b_raw.shape != q_raw.shape[:-1]:
+        raise ValueError("gate shapes disagree with q")
+    for name, s in (("initial_state", initial_state), ("final_state", final_state)):
+        if s is not None and tuple(s.shape) != (B, H, d_k, d_v):
+            raise ValueError(f"{name} must be [B,H,d_k,d_v]")
+    rc = lib().gdn_chunk_prefill_raw(_ptr(q_raw), _ptr(k_raw), _ptr(v), _ptr(a_raw), _ptr(b_raw), float(gate_scale),
+                                     float(norm_eps), _ptr(initial_state), _ptr(out), _ptr(final_state),
+                                     _ptr(cu_seqlens), B, T, H, d_k, d_v, int(chunk), _stream(stream))
+    if rc != 0:
+        raise GdnError(rc, "gdn_chunk_prefill_raw")
+    return out, final_state
 
 
 def gdn_decode_step(q, k, v, log_alpha, beta, state, out, stream=None):

@@ -195,8 +195,29 @@ int gdn_chunk_prefill_snapshots(const void* q, const void* k, const void* v, con
     if (T == 0) return launch_tc(a, reinterpret_cast<cudaStream_t>(stream));
     const size_t need = lean_workspace_bytes(B, T, H, d_k, d_v, false);
     if (!g_workspace || g_workspace_bytes < need) return GDN_ERR_WORKSPACE;
-    return launch_lean(a, g_workspace, g_workspace_bytes, reinterpret_cast<cudaStream_t>(stream), snapshots,
-                       snapshot_every_chunks);
+    LeanOptions opt;
+    opt.snaps = snapshots;
+    opt.snap_every = snapshot_every_chunks;
+    return launch_lean(a, g_workspace, g_workspace_bytes, reinterpret_cast<cudaStream_t>(stream), opt);
+}
+
+int gdn_chunk_prefill_raw(const void* q_raw, const void* k_raw, const void* v, const float* a_raw, const float* b_raw,
+                          float gate_scale, float norm_eps, const float* initial_state, void* out, float* final_state,
+                          const int32_t* cu_seqlens, int B, int T, int H, int d_k, int d_v, int chunk,
+                          gdn_stream_t stream) {
+    const PrefillArgs a = pack(q_raw, k_raw, v, a_raw, b_raw, initial_state, out, final_state, cu_seqlens, B, T, H, d_k, d_v);
+    if (int rc = validate(a, chunk)) return rc;
+    if (!(gate_scale >= 0.f) || !(norm_eps >= 0.f)) return GDN_ERR_INVALID_ARG;
+    if (!tc_supported(d_k, d_v)) return GDN_ERR_UNSUPPORTED;
+    const long tokens = cu_seqlens ? (long)T : (long)B * T;
+    if (tokens == 0) return launch_tc(a, reinterpret_cast<cudaStream_t>(stream));   // only copies the states
+    const size_t need = lean_workspace_bytes(B, T, H, d_k, d_v, cu_seqlens != nullptr);
+    if (!g_workspace || g_workspace_bytes < need) return GDN_ERR_WORKSPACE;
+    LeanOptions opt;
+    opt.raw = true;
+    opt.gate_scale = gate_scale;
+    opt.eps = norm_eps;
+    return launch_lean(a, g_workspace, g_workspace_bytes, reinterpret_cast<cudaStream_t>(stream), opt);
 }
 
 size_t gdn_workspace_bytes(int B, int T, int H, int d_k, int d_v, int packed) {

@@ -41,9 +41,15 @@ bool tc_make_map(CUtensorMap* map, const void* ptr, uint64_t tokens, uint64_t H,
 
 // Two-kernel pipeline (prepare on all SMs, then the chain) using caller-provided scratch.
 size_t lean_workspace_bytes(int B, int T, int H, int d_k, int d_v, bool packed);
-// snaps (optional, batched input only): [B, (T/64)/snap_every, H, d_k, d_v], the state after every snap_every chunks
+struct LeanOptions {
+    float* snaps = nullptr;    // optional (batched input only): [B, (T/64)/snap_every, H, d_k, d_v], the state
+    int snap_every = 1;        //   after every snap_every chunks
+    bool raw = false;          // q, k are raw projections and log_alpha, beta pre-activations: the prepare
+    float gate_scale = 1.f;    //   kernel L2-normalises q, k and applies -softplus(.) * gate_scale and sigmoid(.)
+    float eps = 0.f;           //   (eps under the square root of the norms)
+};
 int launch_lean(const PrefillArgs& a, void* workspace, size_t workspace_bytes, cudaStream_t stream,
-                float* snaps = nullptr, int snap_every = 1);
+                const LeanOptions& opt = LeanOptions());
 int launch_lean_static(const PrefillArgs& a, cudaStream_t stream);   // built-in scratch, allocates nothing
 int lean_query_status();
 void lean_force_segments(int nseg);   // tests only: 0 = automatic plan

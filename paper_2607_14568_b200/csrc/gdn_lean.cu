@@ -136,7 +136,8 @@ constexpr uint32_t PS_T1 = PS_A;                      // ... whose space later h
 constexpr uint32_t PS_TF = PS_A + 64 * LDA * 4;
 constexpr uint32_t PS_Y = PS_TF + 64 * LDA * 4;
 constexpr uint32_t PS_GATES = PS_Y + 32 * LDY * 4;
-constexpr uint32_t PS_BARS = PS_GATES + GATE_FLOATS * 4;
+constexpr uint32_t PS_RN = PS_GATES + GATE_FLOATS * 4;     // raw inputs: 1/|k_i| (64), 1/|q_r| (64)
+constexpr uint32_t PS_BARS = PS_RN + 128 * 4;
 constexpr uint32_t PS_MISC = PS_BARS + 16 * 8;
 constexpr uint32_t PS_TOTAL = PS_MISC + 64;
 constexpr uint32_t PREP_SMEM = PS_TOTAL + 1024;
@@ -152,6 +153,7 @@ struct PrepParams {
     uint8_t* items;
     long nslots;
     int B, T, H;
+    float gate_scale, eps;     // raw inputs only
 };
 
 constexpr uint32_t ID_G = make_idesc(128, 64, kFmtBF16, kFmtBF16, kMajorK, kMajorK);
@@ -179,6 +181,12 @@ __device__ __forceinline__ bool decode_item(const PrepParams& p, long item, int*
     return true;
 }
 
+// RAW: q and k are raw projections and a, beta pre-activations.  The norms and the gating
+// (Section "Batched prefill": per-position kernels around the projections) are folded in here: the
+// inverse row norms scale A, P and the columns of T diag(b e^g), and they ride to the chain kernels
+// inside the gate vectors (e^g / |q| for the output rows, e^{gC-g} / |k| for the state update), so
+// the K and Q tiles themselves are used as they are.
+template <bool RAW>
 __global__ void __launch_bounds__(PREP_THREADS, 3)
 gdn_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k, PrepParams p) {
     extern __shared__ uint8_t smem_raw[];
@@ -188,6 +196,7 @@ gdn_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     float* sTf = reinterpret_cast<float*>(sm + PS_TF);
     float* sY = reinterpret_cast<float*>(sm + PS_Y);
     float* gates = reinterpret_cast<float*>(sm + PS_GATES);
+    float* sRN = reinterpret_cast<float*>(sm + PS_RN);
     volatile uint32_t* sMisc = reinterpret_cast<volatile uint32_t*>(sm + PS_MISC);
     Waiter w{base + PS_BARS, reinterpret_cast<volatile int*>(sm + PS_MISC + 4)};
 
@@ -222,6 +231,29 @@ gdn_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             const int tp = tid;
             const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
             w.wait(PB_GREADY, par);
+            if (RAW) {
+                // inverse L2 norm of row tp of [K;Q] while the G MMA runs (the swizzle only permutes
+                // the 16-byte pieces of a row, so the sum needs no un-swizzling)
+                w.wait(PB_FULL, par);
+                const uint32_t tile = base + PS_KQ + (uint32_t)(tp >> 6) * 8192 + (uint32_t)(tp & 63) * 128;
+                float s0 = 0.f, s1 = 0.f;
+#pragma unroll
+                for (int cgi = 0; cgi < 16; ++cgi) {
+                    const uint32_t addr = tile + (uint32_t)(cgi >> 3) * 16384 + (uint32_t)(((cgi & 7) ^ (tp & 7)) << 4);
+                    uint32_t u[4];
+                    asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
+                                 : "=r"(u[0]), "=r"(u[1]), "=r"(u[2]), "=r"(u[3]) : "r"(addr));
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const float lo = __uint_as_float(u[e] << 16), hi = __uint_as_float(u[e] & 0xffff0000u);
+                        s0 = fmaf(lo, lo, s0);
+                        s1 = fmaf(hi, hi, s1);
+                    }
+                }
+                const float ss = s0 + s1 + p.eps;
+                sRN[tp] = ss > 0.f ? 1.0f / sqrtf(ss) : 0.f;
+                named_bar_sync(1, 128);
+            }
             w.wait(PB_G, par);
             tc_fence_after_sync();
             // ---- step b1: decay masks on G = [K;Q] K^T ----
@@ -229,6 +261,7 @@ gdn_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                 const int r = tp & 63;
                 const float gr = gates[r];
                 const float br = gates[64 + r];
+                const float rnr = RAW ? sRN[tp] : 1.f;        // 1/|k_r| for the A rows, 1/|q_r| for the P rows
                 const bool is_a = tp < 64;
                 const int rmax = 32 * (warp & 1) + 31;
                 const uint32_t pimg = base + PS_KQ + 8192;   // the Q_lo sub-tile is dead once G is complete
@@ -246,6 +279,11 @@ gdn_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                             y[4 * i4 + 1] = ex2(gr - gi.y) * __uint_as_float(x[4 * i4 + 1]);
                             y[4 * i4 + 2] = ex2(gr - gi.z) * __uint_as_float(x[4 * i4 + 2]);
                             y[4 * i4 + 3] = ex2(gr - gi.w) * __uint_as_float(x[4 * i4 + 3]);
+                            if (RAW) {
+                                const float4 rk = *reinterpret_cast<const float4*>(sRN + 32 * hh + 4 * i4);
+                                y[4 * i4 + 0] *= rnr * rk.x; y[4 * i4 + 1] *= rnr * rk.y;
+                                y[4 * i4 + 2] *= rnr * rk.z; y[4 * i4 + 3] *= rnr * rk.w;
+                            }
                         }
                         if (is_a) {
 #pragma unroll
@@ -394,7 +432,7 @@ gdn_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             // ---- step b3 operands: row i = cc of (T diag(b e^g))^T (shared) and (T diag(b))^T (scratch) ----
             {
                 const int cc = tp & 63, half = tp >> 6;
-                const float b = gates[64 + cc], bg = b * gates[128 + cc];
+                const float b = gates[64 + cc], bg = b * gates[128 + cc] * (RAW ? sRN[cc] : 1.f);
                 float t[32];
 #pragma unroll
                 for (int i = 0; i < 32; ++i)
@@ -418,8 +456,14 @@ gdn_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             named_bar_sync(1, 128);
             if (tp == 0) { bulk_store(out_item + IT_T2, base + PS_A + 8192, 8192); bulk_commit(); }
             // ---- step b3 result: -W^T image to scratch; gate vectors to scratch ----
-            if (tp < GATE_FLOATS / 4)
-                *reinterpret_cast<float4*>(out_item + IT_GATES + tp * 16) = *reinterpret_cast<const float4*>(gates + 4 * tp);
+            if (tp < GATE_FLOATS / 4) {
+                float4 gv = *reinterpret_cast<const float4*>(gates + 4 * tp);
+                if (RAW && tp >= 32 && tp < 64) {      // e^g -> e^g / |q|   and   e^{gC-g} -> e^{gC-g} / |k|
+                    const float4 rn = *reinterpret_cast<const float4*>(sRN + (tp < 48 ? 64 + 4 * (tp - 32) : 4 * (tp - 48)));
+                    gv.x *= rn.x; gv.y *= rn.y; gv.z *= rn.z; gv.w *= rn.w;
+                }
+                *reinterpret_cast<float4*>(out_item + IT_GATES + tp * 16) = gv;
+            }
             w.wait(PB_W, par);
             tc_fence_after_sync();
 #pragma unroll
@@ -478,6 +522,10 @@ gdn_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             float x = 0.f, y = 0.f, b0 = 0.f, b1 = 0.f;
             if (r0 < R) { const size_t o = (size_t)(tok + r0) * H + h; x = __ldg(p.a + o); b0 = __ldg(p.beta + o); }
             if (r1 < R) { const size_t o = (size_t)(tok + r1) * H + h; y = __ldg(p.a + o); b1 = __ldg(p.beta + o); }
+            if (RAW) {   // log gate = -softplus(a) * scale, beta = sigmoid(b); padding rows stay the identity token
+                if (r0 < R) { x = -(fmaxf(x, 0.f) + log1pf(expf(-fabsf(x)))) * p.gate_scale; b0 = 1.0f / (1.0f + expf(-b0)); }
+                if (r1 < R) { y = -(fmaxf(y, 0.f) + log1pf(expf(-fabsf(y)))) * p.gate_scale; b1 = 1.0f / (1.0f + expf(-b1)); }
+            }
 #pragma unroll
             for (int d = 1; d < 32; d <<= 1) {
                 const float xu = __shfl_up_sync(0xffffffffu, x, d);
@@ -1222,7 +1270,9 @@ size_t lean_workspace_bytes(int B, int T, int H, int d_k, int d_v, bool packed) 
 }
 
 int launch_lean(const PrefillArgs& a, void* workspace, size_t workspace_bytes, cudaStream_t stream,
-                float* snaps, int snap_every) {
+                const LeanOptions& opt) {
+    float* const snaps = opt.snaps;
+    const int snap_every = opt.snap_every;
     if (!tc_supported(a.d_k, a.d_v)) return GDN_ERR_UNSUPPORTED;
     if (a.H > 65535 || a.B > 4095) return GDN_ERR_UNSUPPORTED;
     const bool packed = a.cu_seqlens != nullptr;
@@ -1240,7 +1290,8 @@ int launch_lean(const PrefillArgs& a, void* workspace, size_t workspace_bytes, c
             cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
             return GDN_ERR_CUDA;
     }
-    if (cudaFuncSetAttribute(gdn_prep_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)PREP_SMEM) != cudaSuccess ||
+    if (cudaFuncSetAttribute(gdn_prep_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)PREP_SMEM) != cudaSuccess ||
+        cudaFuncSetAttribute(gdn_prep_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)PREP_SMEM) != cudaSuccess ||
         cudaFuncSetAttribute(gdn_chain_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)CHAIN_SMEM) != cudaSuccess ||
         cudaFuncSetAttribute(gdn_chain_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)CHAIN_SMEM) != cudaSuccess ||
         cudaFuncSetAttribute(gdn_summary_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SUM_SMEM) != cudaSuccess ||
@@ -1250,11 +1301,12 @@ int launch_lean(const PrefillArgs& a, void* workspace, size_t workspace_bytes, c
     const long nslots = (long)(tokens >> 6) + a.B;
     const long nitems = nslots * a.H;
     // ---- state-independent steps, every (chunk, head) ----
-    PrepParams pp{a.log_alpha, a.beta, a.cu_seqlens, ws, nslots, a.B, a.T, a.H};
+    PrepParams pp{a.log_alpha, a.beta, a.cu_seqlens, ws, nslots, a.B, a.T, a.H, opt.gate_scale, opt.eps};
     const int pgrid = (int)(nitems < 3L * num_sms ? nitems : 3L * num_sms);
     auto mark = [&](int i) { if (g_lean_timing && g_lean_events[i]) cudaEventRecord(g_lean_events[i], stream); };
     mark(0);
-    gdn_prep_kernel<<<pgrid, PREP_THREADS, PREP_SMEM, stream>>>(mq, mk, pp);
+    if (opt.raw) gdn_prep_kernel<true><<<pgrid, PREP_THREADS, PREP_SMEM, stream>>>(mq, mk, pp);
+    else gdn_prep_kernel<false><<<pgrid, PREP_THREADS, PREP_SMEM, stream>>>(mq, mk, pp);
     count_launch();
     if (cudaGetLastError() != cudaSuccess) return GDN_ERR_CUDA;
     mark(1);
@@ -1374,7 +1426,8 @@ int launch_lean_static(const PrefillArgs& a, cudaStream_t stream) {
         int sms = 0;
         if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
             return GDN_ERR_CUDA;
-        if (cudaFuncSetAttribute(gdn_prep_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)PREP_SMEM) != cudaSuccess ||
+        if (cudaFuncSetAttribute(gdn_prep_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)PREP_SMEM) != cudaSuccess ||
+        cudaFuncSetAttribute(gdn_prep_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)PREP_SMEM) != cudaSuccess ||
             cudaFuncSetAttribute(gdn_chain_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)CHAIN_SMEM) != cudaSuccess)
             return GDN_ERR_CUDA;
         sms_of_device[dev] = sms;
@@ -1387,8 +1440,8 @@ int launch_lean_static(const PrefillArgs& a, cudaStream_t stream) {
         return GDN_ERR_CUDA;
     const long nitems = (long)nslots * a.H;
     const long cap = 3L * sms_of_device[dev];
-    PrepParams pp{a.log_alpha, a.beta, a.cu_seqlens, ws, (long)nslots, a.B, a.T, a.H};
-    gdn_prep_kernel<<<(int)(nitems < cap ? nitems : cap), PREP_THREADS, PREP_SMEM, stream>>>(mq, mk, pp);
+    PrepParams pp{a.log_alpha, a.beta, a.cu_seqlens, ws, (long)nslots, a.B, a.T, a.H, 1.f, 0.f};
+    gdn_prep_kernel<false><<<(int)(nitems < cap ? nitems : cap), PREP_THREADS, PREP_SMEM, stream>>>(mq, mk, pp);
     count_launch();
     if (cudaGetLastError() != cudaSuccess) return GDN_ERR_CUDA;
     const int nch = packed ? 1 : (a.T + C - 1) / C;            // one segment: the whole sequence
