@@ -191,7 +191,10 @@ int gdn_chunk_prefill_raw(const void* q_raw, const void* k_raw, const void* v,
  * delta-rule scan for the recurrent layers" -- and leave their results in the scratch for the
  * chain kernel; this is the faster path.  The scratch stays owned by the caller, is 256-byte
  * aligned device memory, must outlive every call that uses it, and is shared by all calls
- * (calls on different streams must not overlap).  gdn_set_workspace(NULL, 0) removes it.
+ * (calls on different streams must not overlap).  gdn_set_workspace zeroes the first 256 bytes
+ * with a synchronous cudaMemset (a work counter that every call leaves at zero again; the caller
+ * must not write there between calls) and returns GDN_ERR_CUDA if that fails; a pointer that is
+ * not 256-byte aligned gives GDN_ERR_UNSUPPORTED.  gdn_set_workspace(NULL, 0) removes it.
  * `packed` is 1 when cu_seqlens will be passed (T = total tokens), else 0.
  * gdn_workspace_bytes returns 0 for sizes the tensor-core path does not support.
  */

@@ -226,8 +226,13 @@ size_t gdn_workspace_bytes(int B, int T, int H, int d_k, int d_v, int packed) {
 
 int gdn_set_workspace(void* device_ptr, size_t bytes) {
     if (device_ptr && (reinterpret_cast<uintptr_t>(device_ptr) & 255u)) return GDN_ERR_UNSUPPORTED;
-    g_workspace = device_ptr;
-    g_workspace_bytes = device_ptr ? bytes : 0;
+    g_workspace = nullptr;
+    g_workspace_bytes = 0;
+    if (device_ptr && bytes >= 256) {
+        if (int rc = lean_init_workspace(device_ptr)) return rc;
+        g_workspace = device_ptr;
+        g_workspace_bytes = bytes;
+    }
     return GDN_OK;
 }
 

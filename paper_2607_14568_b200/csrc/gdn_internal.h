@@ -41,6 +41,7 @@ bool tc_make_map(CUtensorMap* map, const void* ptr, uint64_t tokens, uint64_t H,
 
 // Two-kernel pipeline (prepare on all SMs, then the chain) using caller-provided scratch.
 size_t lean_workspace_bytes(int B, int T, int H, int d_k, int d_v, bool packed);
+int lean_init_workspace(void* workspace);   // zeroes the header of a newly provided workspace (synchronous)
 struct LeanOptions {
     float* snaps = nullptr;    // optional (batched input only): [B, (T/64)/snap_every, H, d_k, d_v], the state
     int snap_every = 1;        //   after every snap_every chunks

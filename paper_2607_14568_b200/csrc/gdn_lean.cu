@@ -58,7 +58,7 @@ constexpr uint32_t IT_GATES = 32768;  //  1280: g log2e | beta | e^g | e^{gC-g} 
 constexpr uint32_t GATE_FLOATS = 320;
 constexpr uint32_t ITEM_BYTES = 34048;
 
-constexpr uint32_t LDA = 68, LDY = 36;
+constexpr uint32_t LDA = 68, LDY = 32;
 
 struct Waiter {
     uint32_t bars;              // shared address of barrier 0
@@ -131,10 +131,11 @@ __device__ __forceinline__ SeqInfo seq_info(const int32_t* cu, int n, int T) {
 // prepare kernel
 // =====================================================================================
 constexpr uint32_t PS_KQ = 0;                         // [K_lo | Q_lo | K_hi | Q_hi]
-constexpr uint32_t PS_A = 32768;                      // fp32 A [64][68] ...
-constexpr uint32_t PS_T1 = PS_A;                      // ... whose space later holds the (T diag(b e^g))^T image
-constexpr uint32_t PS_TF = PS_A + 64 * LDA * 4;
-constexpr uint32_t PS_Y = PS_TF + 64 * LDA * 4;
+constexpr uint32_t PS_A = 32768;                      // fp32 A [64][68], turned into T = (I + A)^{-1} in place;
+                                                      // later the staging space of the -W^T image
+constexpr uint32_t PS_T1 = PS_KQ + 24576;             // (T diag(b e^g))^T image over the Q_hi tile (dead after G)
+constexpr uint32_t PS_T2 = PS_KQ + 8192;              // (T diag(b))^T image over the Q_lo tile, after the P image
+constexpr uint32_t PS_Y = PS_A + 64 * LDA * 4;
 constexpr uint32_t PS_GATES = PS_Y + 32 * LDY * 4;
 constexpr uint32_t PS_RN = PS_GATES + GATE_FLOATS * 4;     // raw inputs: 1/|k_i| (64), 1/|q_r| (64)
 constexpr uint32_t PS_BARS = PS_RN + 128 * 4;
@@ -144,7 +145,7 @@ constexpr uint32_t PREP_SMEM = PS_TOTAL + 1024;
 constexpr int PREP_THREADS = 192;
 constexpr uint32_t PT_COLS = 64;
 
-enum PBar : uint32_t { PB_FULL = 0, PB_G, PB_W, PB_TREADY, PB_GREADY, PB_DONE };
+enum PBar : uint32_t { PB_FULL = 0, PB_G, PB_W, PB_TREADY, PB_GREADY, PB_DONE, PB_KQFREE, PB_ITEM };
 
 struct PrepParams {
     const float* a;
@@ -154,6 +155,7 @@ struct PrepParams {
     long nslots;
     int B, T, H;
     float gate_scale, eps;     // raw inputs only
+    int* ticket;               // {next item, CTAs done}: both zero before the launch, both zero again after it
 };
 
 constexpr uint32_t ID_G = make_idesc(128, 64, kFmtBF16, kFmtBF16, kMajorK, kMajorK);
@@ -187,13 +189,13 @@ __device__ __forceinline__ bool decode_item(const PrepParams& p, long item, int*
 // inside the gate vectors (e^g / |q| for the output rows, e^{gC-g} / |k| for the state update), so
 // the K and Q tiles themselves are used as they are.
 template <bool RAW>
-__global__ void __launch_bounds__(PREP_THREADS, 3)
+__global__ void __launch_bounds__(PREP_THREADS, 4)
 gdn_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k, PrepParams p) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* sm = smem_raw + (base - smem_u32(smem_raw));
     float* sA = reinterpret_cast<float*>(sm + PS_A);
-    float* sTf = reinterpret_cast<float*>(sm + PS_TF);
+    float* sTf = sA;       // the solve overwrites A block by block
     float* sY = reinterpret_cast<float*>(sm + PS_Y);
     float* gates = reinterpret_cast<float*>(sm + PS_GATES);
     float* sRN = reinterpret_cast<float*>(sm + PS_RN);
@@ -205,6 +207,7 @@ gdn_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     if (tid == 0) {
         mbar_init(w.bar(PB_FULL), 1); mbar_init(w.bar(PB_G), 1); mbar_init(w.bar(PB_W), 1);
         mbar_init(w.bar(PB_TREADY), 128); mbar_init(w.bar(PB_GREADY), 32); mbar_init(w.bar(PB_DONE), 128);
+        mbar_init(w.bar(PB_KQFREE), 1); mbar_init(w.bar(PB_ITEM), 1);
         sMisc[1] = 0;
         fence_mbar_init();
     }
@@ -217,12 +220,31 @@ gdn_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     tc_fence_after_sync();
     const uint32_t tmem = sMisc[0];
 
+    // Items are handed out through a global ticket: the time per item differs between SMs by a
+    // quarter, so a fixed assignment would leave the fast ones idle at the end.  The issuing thread
+    // draws the ticket one item ahead and publishes it in shared memory (slot it & 1, barrier PB_ITEM).
     const long nitems = p.nslots * H;
+    int nh = 0, nR = 0;      // issuing thread: head, first token of the item it drew last
+    long ntok = 0;
+    auto draw = [&]() -> int {           // next ticket that names a used slot, or -1
+        while (true) {
+            const int t = atomicAdd(p.ticket, 1);
+            if (t >= nitems) return -1;
+            if (decode_item(p, t, &nh, &ntok, &nR)) return t;
+        }
+    };
+    if (warp == 4 && lane == 0) {
+        sMisc[2] = (uint32_t)draw();
+        mbar_arrive(w.bar(PB_ITEM));
+    }
     int it = 0;     // items this CTA has processed (barrier phases)
-    for (long item = blockIdx.x; item < nitems; item += gridDim.x) {
+    while (true) {
+        w.wait(PB_ITEM, it & 1);
+        const long item = (int)sMisc[2 + (it & 1)];
+        if (item < 0 || *w.abort_flag) break;
         int h, R;
         long tok;
-        if (!decode_item(p, item, &h, &tok, &R)) continue;   // unused slot (uniform for the CTA)
+        decode_item(p, item, &h, &tok, &R);
         uint8_t* out_item = p.items + (size_t)item * ITEM_BYTES;
         const uint32_t par = it & 1;
 
@@ -325,7 +347,6 @@ gdn_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             if (tp < 64) {   // level 0: four 16x16 diagonal blocks, one column per thread
                 const int I = tp >> 4, cc = tp & 15;
                 const float* Ab = sA + (16 * I) * LDA + 16 * I;
-                float* Tb = sTf + (16 * I) * LDA + 16 * I;
                 float xs[16];
 #pragma unroll
                 for (int r = 0; r < 16; ++r) {
@@ -339,8 +360,13 @@ gdn_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                         if (4 * i4 + 3 < r) acc1 = fmaf(a4.w, xs[4 * i4 + 3], acc1);
                     }
                     xs[r] = ((r == cc) ? 1.f : 0.f) - (acc0 + acc1);
-                    Tb[r * LDA + cc] = xs[r];
                 }
+                named_bar_sync(1, 128);                    // every column has read the block: overwrite it
+                float* Tb = sA + (16 * I) * LDA + 16 * I;
+#pragma unroll
+                for (int r = 0; r < 16; ++r) Tb[r * LDA + cc] = xs[r];
+            } else {
+                named_bar_sync(1, 128);
             }
             named_bar_sync(1, 128);
             // The merges are small fp32 products out of shared memory.  A warp owns 8 rows and a lane one
@@ -428,6 +454,7 @@ gdn_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
 #pragma unroll
                 for (int x = 0; x < 8; ++x) sTf[(32 + r0 + x) * LDA + c] = -acc[x];
             }
+            if (tp == 0) bulk_wait_read_all();                 // the P image has left the Q_lo tile
             named_bar_sync(1, 128);
             // ---- step b3 operands: row i = cc of (T diag(b e^g))^T (shared) and (T diag(b))^T (scratch) ----
             {
@@ -447,14 +474,14 @@ gdn_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                         p2[e] = pack_bf16(t0 * b, t1 * b);
                     }
                     st_shared_v4(base + PS_T1 + swz(cc, 4 * half + ch), p1[0], p1[1], p1[2], p1[3]);
-                    st_shared_v4(base + PS_A + 8192 + swz(cc, 4 * half + ch), p2[0], p2[1], p2[2], p2[3]);
+                    st_shared_v4(base + PS_T2 + swz(cc, 4 * half + ch), p2[0], p2[1], p2[2], p2[3]);
                 }
             }
             fence_proxy_async_smem();
             tc_fence_before_sync();
             mbar_arrive(w.bar(PB_TREADY));
             named_bar_sync(1, 128);
-            if (tp == 0) { bulk_store(out_item + IT_T2, base + PS_A + 8192, 8192); bulk_commit(); }
+            if (tp == 0) { bulk_store(out_item + IT_T2, base + PS_T2, 8192); bulk_commit(); }
             // ---- step b3 result: -W^T image to scratch; gate vectors to scratch ----
             if (tp < GATE_FLOATS / 4) {
                 float4 gv = *reinterpret_cast<const float4*>(gates + 4 * tp);
@@ -466,6 +493,12 @@ gdn_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             }
             w.wait(PB_W, par);
             tc_fence_after_sync();
+            if (tp == 0) {
+                // The tensor core is done with the K tiles and the P and T2 copies have left shared
+                // memory: the tiles of the next item may land while this one is finished.
+                bulk_wait_read_all();
+                mbar_arrive(w.bar(PB_KQFREE));
+            }
 #pragma unroll
             for (int hh = 0; hh < 2; ++hh) {
                 uint32_t x[32];
@@ -477,30 +510,32 @@ gdn_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
 #pragma unroll
                     for (int e = 0; e < 4; ++e)
                         pk[e] = pack_bf16(-__uint_as_float(x[8 * ch + 2 * e]), -__uint_as_float(x[8 * ch + 2 * e + 1]));
-                    st_shared_v4(base + PS_KQ + (tp >> 6) * 16384 + swz(tp & 63, 4 * hh + ch), pk[0], pk[1], pk[2], pk[3]);
+                    st_shared_v4(base + PS_A + (tp >> 6) * 8192 + swz(tp & 63, 4 * hh + ch), pk[0], pk[1], pk[2], pk[3]);
                 }
             }
             fence_proxy_async_smem();
             named_bar_sync(1, 128);
-            if (tp == 0) {                                     // rows 0..63 sit over K_lo, rows 64..127 over K_hi
-                bulk_store(out_item + IT_W, base + PS_KQ, 8192);
-                bulk_store(out_item + IT_W + 8192, base + PS_KQ + 16384, 8192);
+            if (tp == 0) {                                     // staged over the fp32 T, which is dead by now
+                bulk_store(out_item + IT_W, base + PS_A, 16384);
                 bulk_commit();
-                bulk_wait_read_all();                          // P, T2, W staging may now be overwritten
+                bulk_wait_read_all();                          // the staging space may now be overwritten
             }
             tc_fence_before_sync();
             mbar_arrive(w.bar(PB_DONE));
         } else if (warp == 4) {
             // ================= TMA + MMA issue (one thread) =================
             if (lane == 0) {
-                if (it > 0) w.wait(PB_DONE, (it - 1) & 1);          // shared memory and TMEM of the last item are free
-                tc_fence_after_sync();
                 const uint32_t kq = base + PS_KQ, full = w.bar(PB_FULL);
-                mbar_arrive_expect_tx(full, 32768);
-                tma_load_3d(kq, &map_k, 0, h, (int)tok, full);
-                tma_load_3d(kq + 8192, &map_q, 0, h, (int)tok, full);
-                tma_load_3d(kq + 16384, &map_k, 64, h, (int)tok, full);
-                tma_load_3d(kq + 24576, &map_q, 64, h, (int)tok, full);
+                auto load_tiles = [&](int hh, long tk) {
+                    mbar_arrive_expect_tx(full, 32768);
+                    tma_load_3d(kq, &map_k, 0, hh, (int)tk, full);
+                    tma_load_3d(kq + 8192, &map_q, 0, hh, (int)tk, full);
+                    tma_load_3d(kq + 16384, &map_k, 64, hh, (int)tk, full);
+                    tma_load_3d(kq + 24576, &map_q, 64, hh, (int)tk, full);
+                };
+                if (it == 0) load_tiles(h, tok);                    // later items were requested one item ahead
+                else w.wait(PB_DONE, (it - 1) & 1);                 // the accumulator columns of the last item are free
+                tc_fence_after_sync();
                 w.wait(PB_FULL, par);
 #pragma unroll
                 for (uint32_t ks = 0; ks < 8; ++ks) {
@@ -508,6 +543,7 @@ gdn_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                     mma_ss(tmem, make_smem_desc(kq + off, 16, 1024), make_smem_desc(kq + off, 16, 1024), ID_G, ks > 0);
                 }
                 mma_commit(w.bar(PB_G));
+                const int nxt = draw();                             // the atomic's latency hides behind the solve
                 w.wait(PB_TREADY, par);
                 tc_fence_after_sync();
 #pragma unroll
@@ -515,6 +551,13 @@ gdn_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                     mma_ss(tmem, make_smem_desc(kq + ks * 2048, 16384, 1024),
                            make_smem_desc(base + PS_T1 + ks * 2048, 1024, 1024), ID_WU, ks > 0);
                 mma_commit(w.bar(PB_W));
+                // request the tiles of the next item as soon as the K/Q space is free, then publish it
+                if (nxt >= 0) {
+                    w.wait(PB_KQFREE, par);
+                    load_tiles(nh, ntok);
+                }
+                sMisc[2 + ((it + 1) & 1)] = (uint32_t)nxt;
+                mbar_arrive(w.bar(PB_ITEM));
             }
         } else {
             // ================= step a: chunk-local cumulative log gate (one warp) =================
@@ -551,6 +594,14 @@ gdn_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     if (warp == 0) {
         tc_fence_after_sync();
         tmem_dealloc(tmem, PT_COLS);
+    }
+    if (tid == 0) {      // the last CTA to leave re-arms the ticket for the next launch
+        __threadfence();
+        if (atomicAdd(p.ticket + 1, 1) == (int)gridDim.x - 1) {
+            p.ticket[0] = 0;
+            p.ticket[1] = 0;
+            __threadfence();
+        }
     }
 }
 
@@ -1254,11 +1305,18 @@ static void plan_split(int B, int T, int H, int d_v, bool packed, int num_sms, i
 }
 constexpr int kMaxSeg = 16;
 
+constexpr size_t kWorkspaceHeader = 256;     // the prepare kernel's item ticket lives in front of the items
+
+// The ticket must read zero before the first launch; every launch leaves it zero again.
+int lean_init_workspace(void* workspace) {
+    return cudaMemset(workspace, 0, kWorkspaceHeader) == cudaSuccess ? GDN_OK : GDN_ERR_CUDA;
+}
+
 size_t lean_workspace_bytes(int B, int T, int H, int d_k, int d_v, bool packed) {
     if (!tc_supported(d_k, d_v) || B <= 0 || T < 0 || H <= 0) return 0;
     const size_t tokens = packed ? (size_t)T : (size_t)B * T;
     const size_t slots = (tokens >> 6) + (size_t)B;
-    size_t bytes = slots * H * ITEM_BYTES;
+    size_t bytes = kWorkspaceHeader + slots * H * ITEM_BYTES;
     bytes = (bytes + 255) & ~(size_t)255;
     if (!packed) {
         // split scratch, sized for the largest plan: incoming states, N_seg and M_seg^T per segment
@@ -1297,12 +1355,13 @@ int launch_lean(const PrefillArgs& a, void* workspace, size_t workspace_bytes, c
         cudaFuncSetAttribute(gdn_summary_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SUM_SMEM) != cudaSuccess ||
         cudaFuncSetAttribute(gdn_combine_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)CMB_SMEM) != cudaSuccess)
         return GDN_ERR_CUDA;
-    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    int* ticket = static_cast<int*>(workspace);                      // header, zeroed by lean_init_workspace
+    uint8_t* ws = static_cast<uint8_t*>(workspace) + kWorkspaceHeader;
     const long nslots = (long)(tokens >> 6) + a.B;
     const long nitems = nslots * a.H;
     // ---- state-independent steps, every (chunk, head) ----
-    PrepParams pp{a.log_alpha, a.beta, a.cu_seqlens, ws, nslots, a.B, a.T, a.H, opt.gate_scale, opt.eps};
-    const int pgrid = (int)(nitems < 3L * num_sms ? nitems : 3L * num_sms);
+    PrepParams pp{a.log_alpha, a.beta, a.cu_seqlens, ws, nslots, a.B, a.T, a.H, opt.gate_scale, opt.eps, ticket};
+    const int pgrid = (int)(nitems < 4L * num_sms ? nitems : 4L * num_sms);
     auto mark = [&](int i) { if (g_lean_timing && g_lean_events[i]) cudaEventRecord(g_lean_events[i], stream); };
     mark(0);
     if (opt.raw) gdn_prep_kernel<true><<<pgrid, PREP_THREADS, PREP_SMEM, stream>>>(mq, mk, pp);
@@ -1404,6 +1463,7 @@ int lean_get_timing(float* ms4) {
 // ------------------------------------------------------------------------------------------
 constexpr size_t kStaticScratchBytes = 64ull << 20;            // 64 MiB
 static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+static __device__ int g_static_ticket[2];                      // the prepare kernel's item ticket (zero at load)
 constexpr int kMaxDevices = 64;
 
 int launch_lean_static(const PrefillArgs& a, cudaStream_t stream) {
@@ -1416,6 +1476,7 @@ int launch_lean_static(const PrefillArgs& a, cudaStream_t stream) {
     if (need > kStaticScratchBytes) return GDN_ERR_TOO_LARGE;
     // ---- set-up, once per device: the device address of the built-in scratch ----
     static void* scratch_of_device[kMaxDevices] = {nullptr};
+    static void* ticket_of_device[kMaxDevices] = {nullptr};
     static int sms_of_device[kMaxDevices] = {0};
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return GDN_ERR_CUDA;
@@ -1423,6 +1484,8 @@ int launch_lean_static(const PrefillArgs& a, cudaStream_t stream) {
     if (!scratch_of_device[dev]) {
         void* ptr = nullptr;
         if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || !ptr) return GDN_ERR_CUDA;
+        if (cudaGetSymbolAddress(&ticket_of_device[dev], g_static_ticket) != cudaSuccess || !ticket_of_device[dev])
+            return GDN_ERR_CUDA;
         int sms = 0;
         if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
             return GDN_ERR_CUDA;
@@ -1439,8 +1502,8 @@ int launch_lean_static(const PrefillArgs& a, cudaStream_t stream) {
         !tc_make_map(&mv, a.v, tokens, a.H, a.d_v))
         return GDN_ERR_CUDA;
     const long nitems = (long)nslots * a.H;
-    const long cap = 3L * sms_of_device[dev];
-    PrepParams pp{a.log_alpha, a.beta, a.cu_seqlens, ws, (long)nslots, a.B, a.T, a.H, 1.f, 0.f};
+    const long cap = 4L * sms_of_device[dev];
+    PrepParams pp{a.log_alpha, a.beta, a.cu_seqlens, ws, (long)nslots, a.B, a.T, a.H, 1.f, 0.f, static_cast<int*>(ticket_of_device[dev])};
     gdn_prep_kernel<false><<<(int)(nitems < cap ? nitems : cap), PREP_THREADS, PREP_SMEM, stream>>>(mq, mk, pp);
     count_launch();
     if (cudaGetLastError() != cudaSuccess) return GDN_ERR_CUDA;
