@@ -6,6 +6,7 @@ only the causally valid prefix and zeroes the tail, then a second product with V
 heads share one key/value head by addressing the same K/V block.
 
   attention_causal     the definition, one (query row, head) at a time: softmax over keys 0..i
+  attention_causal_rows  the same definition for a list of (sequence, position, head) triples
   attention_gemm_form  the paper's order of steps: full rectangular score product, masked softmax
                        that normalises the valid prefix and writes exact zeros beyond it, full
                        rectangular product with V
@@ -41,6 +42,19 @@ def attention_causal(q, k, v, scale):
                 s = (kh[: i + 1] @ q[b, i, h]) * float(scale)      # scores of query i against keys 0..i
                 p = np.exp(s - s.max())
                 out[b, i, h] = (p / p.sum()) @ vh[: i + 1]
+    return out
+
+
+def attention_causal_rows(q, k, v, scale, rows):
+    """attention_causal for the listed (b, i, h) triples only: returns [len(rows), d] (full-size spot checks)."""
+    q, k, v = _f64(q), _f64(k), _f64(v)
+    _check(q, k, v)
+    group = q.shape[2] // k.shape[2]
+    out = np.zeros((len(rows), v.shape[3]))
+    for n, (b, i, h) in enumerate(rows):
+        s = (k[b, : i + 1, h // group] @ q[b, i, h]) * float(scale)
+        p = np.exp(s - s.max())
+        out[n] = (p / p.sum()) @ v[b, : i + 1, h // group]
     return out
 
 

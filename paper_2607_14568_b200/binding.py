@@ -52,6 +52,8 @@ def lib():
         L.gdn_chunk_prefill_snapshots.restype = i
         L.gdn_chunk_prefill_raw.argtypes = [vp] * 5 + [ctypes.c_float] * 2 + [vp] * 4 + [i] * 6 + [vp]
         L.gdn_chunk_prefill_raw.restype = i
+        L.gdn_attn_causal_prefill.argtypes = [vp] * 4 + [i] * 5 + [ctypes.c_float, vp]
+        L.gdn_attn_causal_prefill.restype = i
         L.gdn_workspace_bytes.argtypes = [i] * 6
         L.gdn_workspace_bytes.restype = sz
         L.gdn_set_workspace.argtypes = [vp, sz]
@@ -247,6 +249,24 @@ def gdn_chunk_prefill_raw(q_raw, k_raw, v, a_raw, b_raw, gate_scale, norm_eps, i
     if rc != 0:
         raise GdnError(rc, "gdn_chunk_prefill_raw")
     return out, final_state
+
+
+def gdn_attn_causal_prefill(q, k, v, out, scale=None, stream=None):
+    """Causal softmax attention with grouped queries: q, out [B,T,Hq,d], k, v [B,T,Hkv,d] bf16 on the device;
+    scale defaults to 1/sqrt(d).  See include/gdn_attn.h."""
+    bf = torch.bfloat16
+    _check([("q", q, bf), ("k", k, bf), ("v", v, bf), ("out", out, bf)], bf, "cuda")
+    if q.dim() != 4 or k.dim() != 4 or v.shape != k.shape or out.shape != q.shape or q.shape[:2] != k.shape[:2] \
+            or q.shape[3] != k.shape[3]:
+        raise ValueError("q, out [B,T,Hq,d] and k, v [B,T,Hkv,d] expected")
+    B, T, Hq, d = q.shape
+    if scale is None:
+        scale = 1.0 / float(d) ** 0.5
+    rc = lib().gdn_attn_causal_prefill(_ptr(q), _ptr(k), _ptr(v), _ptr(out), int(B), int(T), int(Hq), int(k.shape[2]),
+                                       int(d), float(scale), _stream(stream))
+    if rc != 0:
+        raise GdnError(rc, "gdn_attn_causal_prefill")
+    return out
 
 
 def gdn_decode_step(q, k, v, log_alpha, beta, state, out, stream=None):

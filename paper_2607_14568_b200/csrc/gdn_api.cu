@@ -3,6 +3,7 @@
 #include <atomic>
 
 #include "gdn_internal.h"
+#include "gdn_attn.h"
 
 namespace gdn {
 
@@ -236,7 +237,19 @@ int gdn_set_workspace(void* device_ptr, size_t bytes) {
     return GDN_OK;
 }
 
-int gdn_query_status(void) { return tc_query_status(); }
+int gdn_attn_causal_prefill(const void* q, const void* k, const void* v, void* out, int B, int T, int Hq, int Hkv,
+                            int d, float scale, gdn_stream_t stream) {
+    if (B < 0 || T < 0 || Hq <= 0 || Hkv <= 0 || d <= 0 || !(scale == scale) || scale - scale != 0.f)
+        return GDN_ERR_INVALID_ARG;
+    if ((B > 0 && T > 0) && (!q || !k || !v || !out)) return GDN_ERR_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out)) return GDN_ERR_UNSUPPORTED;
+    return launch_attn(q, k, v, out, B, T, Hq, Hkv, d, scale, reinterpret_cast<cudaStream_t>(stream));
+}
+
+int gdn_query_status(void) {
+    const int s = tc_query_status();      // synchronises the device
+    return s ? s : attn_query_status();
+}
 
 // Not part of the public header: 0 = automatic, 1 = fused kernel only, 2 = two-kernel pipeline only.
 void gdn_debug_force_path(int path) { g_force_path = path; }

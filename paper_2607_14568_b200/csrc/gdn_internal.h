@@ -65,6 +65,12 @@ bool decode_supported(int d_k, int d_v);
 int launch_decode(const void* q, const void* k, const void* v, const float* log_alpha, const float* beta,
                   float* state, void* out, int B, int H, int d_k, int d_v, cudaStream_t stream);
 
+// Causal grouped-query softmax attention (bf16, d = 128).
+bool attn_supported(int Hq, int Hkv, int d);
+int launch_attn(const void* q, const void* k, const void* v, void* out, int B, int T, int Hq, int Hkv, int d,
+                float scale, cudaStream_t stream);
+int attn_query_status();
+
 void count_launch(int n = 1);
 
 }  // namespace gdn
