@@ -399,12 +399,53 @@ def run_decode(args):
                                    "kernel": "gdn_decode_kernel", "algorithmic_bytes": nbytes}}), flush=True)
 
 
+def run_attention(args):
+    """Secondary line: causal grouped-query attention of one attention layer at a prompt tier
+    (attn_10k: T = 10240, 16 query heads on 8 key/value heads, d = 128)."""
+    import torch
+
+    import paper_2607_14568_b200 as gdn
+    from workloads import get_attn_config, make_attn_inputs
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    name = "attn_2k" if args.workload == "attention_2k" else "attn_10k"
+    cfg = get_attn_config(name)
+    q, k, v = (torch.from_numpy(a.view(np.int16)).view(torch.bfloat16).cuda() for a in make_attn_inputs(cfg))
+    out = torch.empty_like(q)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    for _ in range(max(args.warmup, 3)):
+        gdn.gdn_attn_causal_prefill(q, k, v, out, cfg.scale)
+    torch.cuda.synchronize()
+    for a, b in ev:
+        flush.fill_(1)
+        a.record()
+        gdn.gdn_attn_causal_prefill(q, k, v, out, cfg.scale)
+        b.record()
+    torch.cuda.synchronize()
+    assert gdn.gdn_query_status() == 0
+    ms = float(np.mean([a.elapsed_time(b) for a, b in ev]))
+    # algorithmic flops: two products of 2*d flops per (query, visible key) pair and query head
+    flops = cfg.B * cfg.Hq * 2 * (2 * cfg.d) * (cfg.T * (cfg.T + 1) // 2)
+    peaks = measured_peaks()
+    tf = flops / (ms * 1e-3) / 1e12
+    print(json.dumps({"metric": "attn_causal_prefill_tokens_per_s_per_layer", "value": cfg.B * cfg.T / (ms * 1e-3),
+                      "unit": "tokens/s", "n_gpus": 1, "steps": args.steps, "warmup": max(args.warmup, 3),
+                      "ms_per_step": ms, "higher_is_better": True, "dtype": "bf16", "data": "synthetic",
+                      "config": {"workload": name, "B": cfg.B, "T": cfg.T, "Hq": cfg.Hq, "Hkv": cfg.Hkv, "d": cfg.d,
+                                 "l2": "flushed between timed steps (256 MiB write)"},
+                      "gpu_launches": args.steps,
+                      "roofline": {"bound": "tensor", "achieved": tf, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                                   "frac": tf / peaks["bf16_tflops"], "traffic": None, "peak_source": peaks["source"],
+                                   "kernel": "attn_causal_kernel", "algorithmic_flops": flops}}), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=5)
-    ap.add_argument("--workload", default="long", help="long (T=10240, the metric's configuration), short, serving, large")
+    ap.add_argument("--workload", default="long", help="long (T=10240, the metric's configuration), short, serving, large; secondary lines: decode, "
+                    "attention (T=10240), attention_2k")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-workspace", action="store_true", help="run the fused single-kernel path (no scratch)")
     args = ap.parse_args()
@@ -412,6 +453,8 @@ def main():
         run_reference(args)
     elif args.workload == "decode":
         run_decode(args)
+    elif args.workload in ("attention", "attention_2k"):
+        run_attention(args)
     else:
         run_ours(args)
 

@@ -15,7 +15,7 @@
  * Supported: d = 128, Hq a positive multiple of Hkv.  Where the paper writes the score matrix to
  * a buffer (heads x T x T floats), this library keeps 128 x 128 tiles of it in tensor memory only.
  *
- * Returns GDN_OK, GDN_ERR_INVALID_ARG (null or negative arguments, scale not finite),
+ * Returns GDN_OK, GDN_ERR_INVALID_ARG (null or negative arguments, scale negative or not finite),
  * GDN_ERR_UNSUPPORTED (sizes, alignment), GDN_ERR_TOO_LARGE (B*T >= 2^31), GDN_ERR_CUDA.  The call
  * is asynchronous on `stream`, allocates nothing and owns none of its arguments; B = 0 or T = 0
  * is a no-op.  A bounded wait that expires inside the kernel shows up in gdn_query_status().

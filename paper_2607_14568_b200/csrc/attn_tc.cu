@@ -31,27 +31,28 @@ namespace {
 
 using namespace ptx;
 
-constexpr int BM = 128;                 // queries per CTA
+constexpr int BM = 128;                 // queries per tile (two tiles per CTA)
 constexpr int BN = 128;                 // keys per tile
 constexpr int HD = 128;                 // head dimension
-constexpr int ATTN_THREADS = 192;       // warps 0-3 softmax (one thread per query), 4 MMA issue, 5 TMA
+constexpr int ATTN_THREADS = 320;       // warps 0-3 / 4-7: softmax of query tile A / B (thread = query), 8 MMA issue, 9 TMA
 constexpr unsigned long long ATTN_TIMEOUT_NS = 1000000000ull;
 constexpr float RESCALE_THRESHOLD = 8.f;   // in log2 units: P stays below 2^8
 
-// tensor memory columns (512): two score tiles, the output accumulator, two probability tiles
-constexpr uint32_t TM_S0 = 0, TM_O = 256, TM_P0 = 384;
+// tensor memory columns (512): scores of tile A and B (their bf16 probabilities overwrite the first
+// 64 columns of the scores they came from), output accumulators of A and B
+constexpr uint32_t TM_S = 0, TM_O = 256;
 constexpr uint32_t AT_COLS = 512;
 
 // shared memory: a tile is [2 halves of the head dimension][128 rows][64 values], 128-byte rows
 constexpr uint32_t TILE_BYTES = 32768;
-constexpr uint32_t AS_Q = 0, AS_K = TILE_BYTES, AS_V = 3 * TILE_BYTES;          // K, V: two stages each
-constexpr uint32_t AS_BARS = 5 * TILE_BYTES;
+constexpr uint32_t AS_Q = 0, AS_K = 2 * TILE_BYTES, AS_V = 4 * TILE_BYTES;      // Q: A, B; K, V: two stages each
+constexpr uint32_t AS_BARS = 6 * TILE_BYTES;
 constexpr uint32_t AS_MISC = AS_BARS + 24 * 8;
 constexpr uint32_t AS_TOTAL = AS_MISC + 64;
 constexpr uint32_t ATTN_SMEM = AS_TOTAL + 1024;
 
-enum ABar : uint32_t { AB_Q = 0, AB_KFULL0 = 1, AB_KFREE0 = 3, AB_VFULL0 = 5, AB_VFREE0 = 7, AB_SFULL0 = 9,
-                       AB_SFREE0 = 11, AB_PFULL = 13, AB_PVDONE = 14 };
+enum ABar : uint32_t { AB_Q = 0, AB_KFULL0 = 1, AB_KFREE0 = 3, AB_VFULL0 = 5, AB_VFREE0 = 7, AB_SFULL0 = 9 /* A, B */,
+                       AB_PFULL0 = 11 /* A, B */, AB_PVDONE0 = 13 /* A, B */ };
 
 struct AWaiter {
     uint32_t bars;
@@ -84,7 +85,9 @@ struct AttnParams {
 constexpr uint32_t ID_QK = make_idesc(128, 128, kFmtBF16, kFmtBF16, kMajorK, kMajorK);
 constexpr uint32_t ID_PV = make_idesc(128, 128, kFmtBF16, kFmtBF16, kMajorK, kMajorMN);
 
-
+// One CTA owns two neighbouring query tiles A = 2t, B = 2t + 1 of one head.  Both read the same key
+// and value tiles, and their softmax warpgroups alternate: while one turns its scores into
+// probabilities, the tensor core runs P V and the next Q K^T of the other.
 __global__ void __launch_bounds__(ATTN_THREADS, 1)
 attn_causal_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                    const __grid_constant__ CUtensorMap map_v, AttnParams p) {
@@ -96,20 +99,23 @@ attn_causal_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int nqt = (p.T + BM - 1) / BM;
-    const int qt = nqt - 1 - (int)blockIdx.x;              // longest rows of tiles first
+    const int npair = (nqt + 1) / 2;
+    const int t = npair - 1 - (int)blockIdx.x;             // longest rows of tiles first
     const int h = blockIdx.y, b = blockIdx.z;
     const int hk = h / (p.Hq / p.Hkv);                     // the key/value head this query head reads
-    const int ntiles = qt + 1;                             // key tiles 0..qt (the last one is the diagonal)
-    const int tok_q = b * p.T + qt * BM;
+    const bool hasB = (2 * t + 1 < nqt);
+    const int nA = 2 * t + 1;                              // key tiles of A: 0..2t (the last is its diagonal)
+    const int nB = hasB ? 2 * t + 2 : 0;
+    const int ntiles = hasB ? nB : nA;
 
     if (tid == 0) {
         mbar_init(w.bar(AB_Q), 1);
         for (uint32_t s = 0; s < 2; ++s) {
             mbar_init(w.bar(AB_KFULL0 + s), 1); mbar_init(w.bar(AB_KFREE0 + s), 1);
             mbar_init(w.bar(AB_VFULL0 + s), 1); mbar_init(w.bar(AB_VFREE0 + s), 1);
-            mbar_init(w.bar(AB_SFULL0 + s), 1); mbar_init(w.bar(AB_SFREE0 + s), 128);
+            mbar_init(w.bar(AB_SFULL0 + s), 1); mbar_init(w.bar(AB_PFULL0 + s), 128);
+            mbar_init(w.bar(AB_PVDONE0 + s), 1);
         }
-        mbar_init(w.bar(AB_PFULL), 128); mbar_init(w.bar(AB_PVDONE), 1);
         sMisc[1] = 0;
         fence_mbar_init();
     }
@@ -122,131 +128,174 @@ attn_causal_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
     tc_fence_after_sync();
     const uint32_t tmem = sMisc[0];
 
-    if (warp < 4) {
+    if (warp < 8) {
         // =========================== softmax: thread = query row ===========================
-        const int r = tid;                                 // row inside the tile = tensor-memory lane
-        const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
+        const uint32_t X = warp >> 2;                      // 0 = tile A, 1 = tile B
+        const int nX = X ? nB : nA;
+        const int qt = 2 * t + (int)X;
+        const int r = tid & 127;                           // row inside the tile = tensor-memory lane
+        const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
+        const uint32_t ts = tmem + lane_base + TM_S + X * 128, to = tmem + lane_base + TM_O + X * 128;
+        const float c = p.scale_log2e;
         float m_ref = -INFINITY, l = 0.f;
-        for (int j = 0; j < ntiles; ++j) {
-            const uint32_t sb = j & 1;
-            w.wait(AB_SFULL0 + sb, (j >> 1) & 1);
+        for (int j = 0; j < nX; ++j) {
+            // S_X of tile j is complete; so is every earlier MMA of the issuing thread (P V of tile j - 1)
+            w.wait(AB_SFULL0 + X, j & 1);
             tc_fence_after_sync();
-            uint32_t x[4][32];
+            // pass 1: row maximum of the raw scores (c >= 0, so max(c s) = c max(s)); the scores are read
+            // again in pass 2 instead of being kept, so that both passes have registers to overlap their
+            // loads, special-function operations and conversions
+            float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+            {
+                uint32_t x[4][32];
 #pragma unroll
-            for (int q4 = 0; q4 < 4; ++q4) tmem_ld32(tmem + lane_base + TM_S0 + sb * 128 + 32 * q4, x[q4]);
-            tmem_wait_ld();
-            tc_fence_before_sync();
-            mbar_arrive(w.bar(AB_SFREE0 + sb));            // the next-but-one score tile may overwrite this one
-            const bool diag = (j == qt);
-            float mx = -INFINITY;
+                for (int q4 = 0; q4 < 4; ++q4) tmem_ld32(ts + 32 * q4, x[q4]);
+                tmem_wait_ld();
+                if (j == qt) {                             // diagonal tile: keys after the query do not count
 #pragma unroll
-            for (int q4 = 0; q4 < 4; ++q4)
+                    for (int q4 = 0; q4 < 4; ++q4)
 #pragma unroll
-                for (int i = 0; i < 32; ++i) {
-                    float s = __uint_as_float(x[q4][i]) * p.scale_log2e;
-                    if (diag && 32 * q4 + i > r) s = -INFINITY;            // keys after the query
-                    x[q4][i] = __float_as_uint(s);
-                    mx = fmaxf(mx, s);
+                        for (int i = 0; i < 32; ++i)
+                            if (32 * q4 + i > r) x[q4][i] = 0xff800000u;       // -inf
                 }
+#pragma unroll
+                for (int q4 = 0; q4 < 4; ++q4)
+#pragma unroll
+                    for (int i = 0; i < 32; i += 2)
+                        mx4[(i >> 1) & 3] = max3(mx4[(i >> 1) & 3], __uint_as_float(x[q4][i]), __uint_as_float(x[q4][i + 1]));
+            }
+            const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * c;
             // raise the reference maximum only when it is first set or has grown by more than 2^8
             const bool grow = (mx > m_ref + RESCALE_THRESHOLD);
             const float m_new = grow ? mx : m_ref;
             const float alpha = grow ? ex2(m_ref - m_new) : 1.f;           // 0 on the first tile (m_ref = -inf)
             m_ref = m_new;
-            float sum = 0.f;
-            uint32_t pk[64];
+            // pass 2: P = 2^(c s - m) as bf16 over the first 64 columns of the scores it came from; the
+            // next 32 columns are requested before the current 32 are worked on
+            float sum[4] = {0.f, 0.f, 0.f, 0.f};
+            uint32_t xs[2][32];
+            tmem_ld32(ts, xs[0]);
 #pragma unroll
-            for (int q4 = 0; q4 < 4; ++q4)
+            for (int q4 = 0; q4 < 4; ++q4) {
+                tmem_wait_ld();
+                if (q4 < 3) tmem_ld32(ts + 32 * (q4 + 1), xs[(q4 + 1) & 1]);
+                uint32_t pk[16];
 #pragma unroll
-                for (int i = 0; i < 32; i += 2) {
-                    const float p0 = ex2(__uint_as_float(x[q4][i]) - m_new);
-                    const float p1 = ex2(__uint_as_float(x[q4][i + 1]) - m_new);
-                    sum += p0 + p1;
-                    pk[16 * q4 + (i >> 1)] = pack_bf16(p0, p1);
-                }
-            l = l * alpha + sum;
-            // O and this probability buffer are free once the previous P V product has completed
-            if (j > 0) {
-                w.wait(AB_PVDONE, (j - 1) & 1);
-                tc_fence_after_sync();
-                if (__any_sync(0xffffffffu, grow)) {       // rescale the accumulator rows of this warp
-#pragma unroll
-                    for (int q4 = 0; q4 < 4; ++q4) {
-                        uint32_t o[32];
-                        tmem_ld32(tmem + lane_base + TM_O + 32 * q4, o);
-                        tmem_wait_ld();
-#pragma unroll
-                        for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
-                        tmem_st32(tmem + lane_base + TM_O + 32 * q4, o);
+                for (int i = 0; i < 16; ++i) {
+                    const int e = 32 * q4 + 2 * i;
+                    float p0 = ex2(fmaf(__uint_as_float(xs[q4 & 1][2 * i]), c, -m_new));
+                    float p1 = ex2(fmaf(__uint_as_float(xs[q4 & 1][2 * i + 1]), c, -m_new));
+                    if (j == qt) {                         // exact zeros after the query's own position
+                        if (e > r) p0 = 0.f;
+                        if (e + 1 > r) p1 = 0.f;
                     }
+                    sum[i & 1] += p0;
+                    sum[2 + (i & 1)] += p1;
+                    pk[i] = pack_bf16(p0, p1);
                 }
+                tmem_st16(ts + 16 * q4, pk);
             }
+            const float sum0 = sum[0] + sum[1], sum1 = sum[2] + sum[3];
+            l = l * alpha + (sum0 + sum1);
+            if (j > 0 && __any_sync(0xffffffffu, grow)) {   // rescale the accumulator rows of this warp
 #pragma unroll
-            for (int q2 = 0; q2 < 2; ++q2) {
-                uint32_t o[32];
+                for (int q4 = 0; q4 < 4; ++q4) {
+                    uint32_t o[32];
+                    tmem_ld32(to + 32 * q4, o);
+                    tmem_wait_ld();
 #pragma unroll
-                for (int i = 0; i < 32; ++i) o[i] = pk[32 * q2 + i];
-                tmem_st32(tmem + lane_base + TM_P0 + sb * 64 + 32 * q2, o);
+                    for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+                    tmem_st32(to + 32 * q4, o);
+                }
             }
             tmem_wait_st();
             tc_fence_before_sync();
-            mbar_arrive(w.bar(AB_PFULL));
+            mbar_arrive(w.bar(AB_PFULL0 + X));
         }
         // ---- epilogue: O / l -> bf16 -> global (one 256-byte row per thread) ----
-        w.wait(AB_PVDONE, (ntiles - 1) & 1);
-        tc_fence_after_sync();
-        const float inv = 1.0f / l;
-        const int row = qt * BM + r;
-        __nv_bfloat16* dst = p.out + ((size_t)(b * p.T + row) * p.Hq + h) * HD;
+        if (nX > 0) {
+            w.wait(AB_PVDONE0 + X, 0);
+            tc_fence_after_sync();
+            const float inv = 1.0f / l;
+            const int row = qt * BM + r;
+            __nv_bfloat16* dst = p.out + ((size_t)(b * p.T + row) * p.Hq + h) * HD;
 #pragma unroll
-        for (int q4 = 0; q4 < 4; ++q4) {
-            uint32_t o[32];
-            tmem_ld32(tmem + lane_base + TM_O + 32 * q4, o);
-            tmem_wait_ld();
-            if (row < p.T) {
+            for (int q4 = 0; q4 < 4; ++q4) {
+                uint32_t o[32];
+                tmem_ld32(to + 32 * q4, o);
+                tmem_wait_ld();
+                if (row < p.T) {
 #pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    uint4 val;
-                    val.x = pack_bf16(__uint_as_float(o[8 * c + 0]) * inv, __uint_as_float(o[8 * c + 1]) * inv);
-                    val.y = pack_bf16(__uint_as_float(o[8 * c + 2]) * inv, __uint_as_float(o[8 * c + 3]) * inv);
-                    val.z = pack_bf16(__uint_as_float(o[8 * c + 4]) * inv, __uint_as_float(o[8 * c + 5]) * inv);
-                    val.w = pack_bf16(__uint_as_float(o[8 * c + 6]) * inv, __uint_as_float(o[8 * c + 7]) * inv);
-                    *reinterpret_cast<uint4*>(dst + 32 * q4 + 8 * c) = val;
+                    for (int cc = 0; cc < 4; ++cc) {
+                        uint4 val;
+                        val.x = pack_bf16(__uint_as_float(o[8 * cc + 0]) * inv, __uint_as_float(o[8 * cc + 1]) * inv);
+                        val.y = pack_bf16(__uint_as_float(o[8 * cc + 2]) * inv, __uint_as_float(o[8 * cc + 3]) * inv);
+                        val.z = pack_bf16(__uint_as_float(o[8 * cc + 4]) * inv, __uint_as_float(o[8 * cc + 5]) * inv);
+                        val.w = pack_bf16(__uint_as_float(o[8 * cc + 6]) * inv, __uint_as_float(o[8 * cc + 7]) * inv);
+                        *reinterpret_cast<uint4*>(dst + 32 * q4 + 8 * cc) = val;
+                    }
                 }
             }
         }
-    } else if (warp == 4) {
+    } else if (warp == 8) {
         // =========================== MMA issue (one thread) ===========================
         if (lane == 0) {
-            const uint32_t qa = base + AS_Q;
-            auto issue_qk = [&](int j) {                   // S[j & 1] = Q K_j^T
-                const uint32_t s = j & 1, ka = base + AS_K + s * TILE_BYTES;
-                w.wait(AB_KFULL0 + s, (j >> 1) & 1);
-                if (j >= 2) w.wait(AB_SFREE0 + s, ((j >> 1) - 1) & 1);
-                tc_fence_after_sync();
+            // operand descriptors are built once: issuing costs tens of nanoseconds per instruction and
+            // sits on each tile's softmax -> P V -> Q K^T chain
+            const uint64_t dq0 = make_smem_desc(base + AS_Q, 16, 1024), dk0 = make_smem_desc(base + AS_K, 16, 1024);
+            const uint64_t dv0 = make_smem_desc(base + AS_V, 16384, 1024);
+            auto issue_qk = [&](uint32_t X, int j) {       // S_X = Q_X K_j^T
+                const uint64_t dq = dq0 + ((uint64_t)(X * TILE_BYTES) >> 4), dk = dk0 + ((uint64_t)((j & 1) * TILE_BYTES) >> 4);
 #pragma unroll
                 for (uint32_t ks = 0; ks < 8; ++ks) {
-                    const uint32_t off = (ks >> 2) * 16384 + (ks & 3) * 32;
-                    mma_ss(tmem + TM_S0 + s * 128, make_smem_desc(qa + off, 16, 1024), make_smem_desc(ka + off, 16, 1024),
-                           ID_QK, ks > 0);
+                    const uint64_t off = ((ks >> 2) * 16384 + (ks & 3) * 32) >> 4;   // the address field counts 16 bytes
+                    mma_ss(tmem + TM_S + X * 128, dq + off, dk + off, ID_QK, ks > 0);
                 }
-                mma_commit(w.bar(AB_SFULL0 + s));
-                mma_commit(w.bar(AB_KFREE0 + s));
+                mma_commit(w.bar(AB_SFULL0 + X));
+            };
+            auto issue_pv = [&](uint32_t X, int j) {       // O_X += P_X V_j, 16 keys per step
+                const uint64_t dv = dv0 + ((uint64_t)((j & 1) * TILE_BYTES) >> 4);
+#pragma unroll
+                for (uint32_t ks = 0; ks < 8; ++ks)
+                    mma_ts(tmem + TM_O + X * 128, tmem + TM_S + X * 128 + ks * 8, dv + ((ks * 2048) >> 4), ID_PV,
+                           (j > 0 || ks > 0) ? 1u : 0u);
             };
             w.wait(AB_Q, 0);
-            issue_qk(0);
+            w.wait(AB_KFULL0, 0);
+            tc_fence_after_sync();
+            issue_qk(0, 0);
+            if (hasB) issue_qk(1, 0);
+            mma_commit(w.bar(AB_KFREE0));
             for (int j = 0; j < ntiles; ++j) {
-                if (j + 1 < ntiles) issue_qk(j + 1);
-                const uint32_t s = j & 1, va = base + AS_V + s * TILE_BYTES;
+                const uint32_t s = j & 1, s1 = (j + 1) & 1;
+                const bool more = (j + 1 < ntiles);
                 w.wait(AB_VFULL0 + s, (j >> 1) & 1);
-                w.wait(AB_PFULL, j & 1);
-                tc_fence_after_sync();
-#pragma unroll
-                for (uint32_t ks = 0; ks < 8; ++ks)        // O += P V_j, 16 keys per step
-                    mma_ts(tmem + TM_O, tmem + TM_P0 + s * 64 + ks * 8, make_smem_desc(va + ks * 2048, 16384, 1024),
-                           ID_PV, (j > 0 || ks > 0) ? 1u : 0u);
-                mma_commit(w.bar(AB_PVDONE));
+                if (j < nA) {
+                    w.wait(AB_PFULL0 + 0, j & 1);
+                    tc_fence_after_sync();
+                    issue_pv(0, j);
+                    if (j + 1 < nA) {
+                        w.wait(AB_KFULL0 + s1, ((j + 1) >> 1) & 1);
+                        tc_fence_after_sync();
+                        issue_qk(0, j + 1);
+                    } else {
+                        mma_commit(w.bar(AB_PVDONE0 + 0));
+                    }
+                }
+                if (hasB) {
+                    w.wait(AB_PFULL0 + 1, j & 1);
+                    tc_fence_after_sync();
+                    issue_pv(1, j);
+                    if (more) {
+                        w.wait(AB_KFULL0 + s1, ((j + 1) >> 1) & 1);
+                        tc_fence_after_sync();
+                        issue_qk(1, j + 1);
+                    } else {
+                        mma_commit(w.bar(AB_PVDONE0 + 1));
+                    }
+                }
                 mma_commit(w.bar(AB_VFREE0 + s));
+                if (more) mma_commit(w.bar(AB_KFREE0 + s1));
             }
         }
     } else {
@@ -256,19 +305,23 @@ attn_causal_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             prefetch_tensormap(&map_k);
             prefetch_tensormap(&map_v);
             auto load_tile = [&](uint32_t dst, const CUtensorMap* map, int head, int tok, uint32_t full) {
-                mbar_arrive_expect_tx(full, TILE_BYTES);
                 tma_load_3d(dst, map, 0, head, tok, full);
                 tma_load_3d(dst + 8192, map, 0, head, tok + 64, full);
                 tma_load_3d(dst + 16384, map, 64, head, tok, full);
                 tma_load_3d(dst + 24576, map, 64, head, tok + 64, full);
             };
+            const int tok_q = b * p.T + 2 * t * BM;
+            mbar_arrive_expect_tx(w.bar(AB_Q), hasB ? 2 * TILE_BYTES : TILE_BYTES);
             load_tile(base + AS_Q, &map_q, h, tok_q, w.bar(AB_Q));
+            if (hasB) load_tile(base + AS_Q + TILE_BYTES, &map_q, h, tok_q + BM, w.bar(AB_Q));
             for (int j = 0; j < ntiles; ++j) {
                 const uint32_t s = j & 1;
                 const int tok = b * p.T + j * BN;
                 if (j >= 2) w.wait(AB_KFREE0 + s, ((j >> 1) - 1) & 1);
+                mbar_arrive_expect_tx(w.bar(AB_KFULL0 + s), TILE_BYTES);
                 load_tile(base + AS_K + s * TILE_BYTES, &map_k, hk, tok, w.bar(AB_KFULL0 + s));
                 if (j >= 2) w.wait(AB_VFREE0 + s, ((j >> 1) - 1) & 1);
+                mbar_arrive_expect_tx(w.bar(AB_VFULL0 + s), TILE_BYTES);
                 load_tile(base + AS_V + s * TILE_BYTES, &map_v, hk, tok, w.bar(AB_VFULL0 + s));
             }
             if (*w.abort_flag) {
@@ -312,11 +365,11 @@ int launch_attn(const void* q, const void* k, const void* v, void* out, int B, i
     if (!tc_make_map(&mq, q, tokens, Hq, d) || !tc_make_map(&mk, k, tokens, Hkv, d) ||
         !tc_make_map(&mv, v, tokens, Hkv, d))
         return GDN_ERR_CUDA;
+    AttnParams p{static_cast<__nv_bfloat16*>(out), B, T, Hq, Hkv, scale * 1.4426950408889634f};
+    dim3 grid(((T + BM - 1) / BM + 1) / 2, Hq, B);
     if (cudaFuncSetAttribute(attn_causal_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ATTN_SMEM) !=
         cudaSuccess)
         return GDN_ERR_CUDA;
-    AttnParams p{static_cast<__nv_bfloat16*>(out), B, T, Hq, Hkv, scale * 1.4426950408889634f};
-    dim3 grid((T + BM - 1) / BM, Hq, B);
     attn_causal_kernel<<<grid, ATTN_THREADS, ATTN_SMEM, stream>>>(mq, mk, mv, p);
     count_launch();
     return cudaGetLastError() == cudaSuccess ? GDN_OK : GDN_ERR_CUDA;
