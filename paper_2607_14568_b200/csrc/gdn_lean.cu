@@ -849,8 +849,13 @@ gdn_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             // ---- MMA issuer of the sequential chain: v_new and the state update, nothing else ----
             // (issuing costs tens of nanoseconds per instruction; everything off the chain is
             //  issued by a second thread so that it does not sit between two dependent steps)
+            // operand descriptors are built once per stage, outside the dependent chain: the address field
+            // counts 16-byte units, so a k-step is a plain add
+            const uint64_t dW0 = make_smem_desc(base + CS_A + ST_W, 1024, 1024);
+            const uint64_t dK0 = make_smem_desc(base + CS_A + ST_KQ, 16384, 1024);
             for (int c = 0; c < nchunks; ++c) {
-                const uint32_t s = c & 1, sb = base + CS_A + s * STAGE_A;
+                const uint32_t s = c & 1;
+                const uint64_t dW = dW0 + (uint64_t)((s * STAGE_A) >> 4), dK = dK0 + (uint64_t)((s * STAGE_A) >> 4);
                 w.wait_hot(CB_SREADY, c & 1);
                 w.wait_hot(CB_FULLA0 + s, (c >> 1) & 1);
                 w.wait_hot(CB_U, c & 1);                       // U^T of this chunk is in the accumulator
@@ -858,7 +863,7 @@ gdn_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                 stamp(1, c, 0);
 #pragma unroll
                 for (uint32_t ks = 0; ks < 8; ++ks)            // v^T = U^T - S^T W^T
-                    mma_ts(tmem + TM_DV, tmem + TM_SBF + ks * 8, make_smem_desc(sb + ST_W + ks * 2048, 1024, 1024), ID_1, 1);
+                    mma_ts(tmem + TM_DV, tmem + TM_SBF + ks * 8, dW + ks * 128, ID_1, 1);
                 mma_commit(w.bar(CB_V));
                 stamp(1, c, 1);
                 w.wait_hot(CB_VREADY, c & 1);
@@ -866,7 +871,7 @@ gdn_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                 stamp(1, c, 3);
 #pragma unroll
                 for (uint32_t ks = 0; ks < 4; ++ks)            // dS^T = (v e^{gC-g})^T K
-                    mma_ts(tmem + TM_DS, tmem + TM_VT + ks * 8, make_smem_desc(sb + ST_KQ + ks * 2048, 16384, 1024), ID_2, ks > 0);
+                    mma_ts(tmem + TM_DS, tmem + TM_VT + ks * 8, dK + ks * 128, ID_2, ks > 0);
                 mma_commit(w.bar(CB_S));
                 mma_commit(w.bar(CB_FREEA0 + s));
                 stamp(1, c, 4);
@@ -1119,8 +1124,10 @@ gdn_summary_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
             // ---- one MMA issue thread per chain instance (they are independent) ----
             const int inst = (warp == 8) ? 0 : 1;
             if (inst < ninst) {
+                const uint64_t dW0 = make_smem_desc(base + SS_W, 1024, 1024), dK0 = make_smem_desc(base + SS_K, 8192, 1024);
                 for (int c = 0; c < nchunks; ++c) {
                     const uint32_t s = c % SUM_STAGES, sb = base + s * SUM_STAGE;
+                    const uint64_t dW = dW0 + (uint64_t)((s * SUM_STAGE) >> 4), dK = dK0 + (uint64_t)((s * SUM_STAGE) >> 4);
                     w.wait_hot(SB_FULL0 + s, (c / SUM_STAGES) & 1);
                     if (inst == 0) {
                         tc_fence_after_sync();
@@ -1134,14 +1141,14 @@ gdn_summary_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
 #pragma unroll
                     for (uint32_t ks = 0; ks < 8; ++ks)            // v^T = U^T - S^T W^T   (U = 0 for the identity chain)
                         mma_ts(tmem + sum_dv(inst), tmem + sum_ds(inst) + ks * 8,
-                               make_smem_desc(sb + SS_W + ks * 2048, 1024, 1024), ID_1, (inst == 0 || ks > 0) ? 1u : 0u);
+                               dW + ks * 128, ID_1, (inst == 0 || ks > 0) ? 1u : 0u);
                     mma_commit(w.bar(SB_V0 + inst));
                     w.wait_hot(SB_VREADY0 + inst, c & 1);
                     tc_fence_after_sync();
 #pragma unroll
                     for (uint32_t ks = 0; ks < 4; ++ks)            // dS^T = (v e^{gC-g})^T K
                         mma_ts(tmem + sum_ds(inst), tmem + sum_vt(inst) + ks * 8,
-                               make_smem_desc(sb + SS_K + ks * 2048, 8192, 1024), ID_2, ks > 0);
+                               dK + ks * 128, ID_2, ks > 0);
                     mma_commit(w.bar(SB_S0 + inst));
                     mma_commit(w.bar(SB_FREE0 + s));
                 }
