@@ -440,19 +440,24 @@ gdn_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                 named_bar_sync(1, 128);
 #pragma unroll
                 for (int x = 0; x < 8; ++x) acc[x] = 0.f;
-#pragma unroll 2
+                // T22 is lower triangular: row r of it ends at column r.  With the rows dealt out round robin
+                // (this warp owns rows warp, warp + 4, ...) row x of the warp needs the column blocks 0..x only,
+                // the same for every warp: 36 of the 64 (block, row) pairs.
+#pragma unroll
                 for (int i4 = 0; i4 < 8; ++i4) {
                     float yv[4];
 #pragma unroll
                     for (int e = 0; e < 4; ++e) yv[e] = sY[(4 * i4 + e) * LDY + c];
 #pragma unroll
                     for (int x = 0; x < 8; ++x) {
-                        const float4 a4 = *reinterpret_cast<const float4*>(sTf + (32 + r0 + x) * LDA + 32 + 4 * i4);
-                        acc[x] = fmaf(a4.x, yv[0], fmaf(a4.y, yv[1], fmaf(a4.z, yv[2], fmaf(a4.w, yv[3], acc[x]))));
+                        if (x >= i4) {
+                            const float4 a4 = *reinterpret_cast<const float4*>(sTf + (32 + warp + 4 * x) * LDA + 32 + 4 * i4);
+                            acc[x] = fmaf(a4.x, yv[0], fmaf(a4.y, yv[1], fmaf(a4.z, yv[2], fmaf(a4.w, yv[3], acc[x]))));
+                        }
                     }
                 }
 #pragma unroll
-                for (int x = 0; x < 8; ++x) sTf[(32 + r0 + x) * LDA + c] = -acc[x];
+                for (int x = 0; x < 8; ++x) sTf[(32 + warp + 4 * x) * LDA + c] = -acc[x];
             }
             if (tp == 0) bulk_wait_read_all();                 // the P image has left the Q_lo tile
             named_bar_sync(1, 128);
