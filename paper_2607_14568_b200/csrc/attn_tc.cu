@@ -100,8 +100,8 @@ attn_causal_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int nqt = (p.T + BM - 1) / BM;
     const int npair = (nqt + 1) / 2;
-    const int t = npair - 1 - (int)blockIdx.x;             // longest rows of tiles first
-    const int h = blockIdx.y, b = blockIdx.z;
+    const int t = npair - 1 - (int)blockIdx.y;             // CTAs start in x-major order: every head's longest
+    const int h = blockIdx.x, b = blockIdx.z;              // pair of tiles first, the short ones fill the tail
     const int hk = h / (p.Hq / p.Hkv);                     // the key/value head this query head reads
     const bool hasB = (2 * t + 1 < nqt);
     const int nA = 2 * t + 1;                              // key tiles of A: 0..2t (the last is its diagonal)
@@ -357,7 +357,7 @@ int attn_query_status() {
 int launch_attn(const void* q, const void* k, const void* v, void* out, int B, int T, int Hq, int Hkv, int d,
                 float scale, cudaStream_t stream) {
     if (!attn_supported(Hq, Hkv, d)) return GDN_ERR_UNSUPPORTED;
-    if (Hq > 65535 || B > 65535) return GDN_ERR_UNSUPPORTED;
+    if (B > 65535 || ((T + BM - 1) / BM + 1) / 2 > 65535) return GDN_ERR_UNSUPPORTED;
     if (B == 0 || T == 0) return GDN_OK;
     const uint64_t tokens = (uint64_t)B * T;
     if (tokens > 0x7fffffffull) return GDN_ERR_TOO_LARGE;
@@ -366,7 +366,7 @@ int launch_attn(const void* q, const void* k, const void* v, void* out, int B, i
         !tc_make_map(&mv, v, tokens, Hkv, d))
         return GDN_ERR_CUDA;
     AttnParams p{static_cast<__nv_bfloat16*>(out), B, T, Hq, Hkv, scale * 1.4426950408889634f};
-    dim3 grid(((T + BM - 1) / BM + 1) / 2, Hq, B);
+    dim3 grid(Hq, ((T + BM - 1) / BM + 1) / 2, B);
     if (cudaFuncSetAttribute(attn_causal_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ATTN_SMEM) !=
         cudaSuccess)
         return GDN_ERR_CUDA;
