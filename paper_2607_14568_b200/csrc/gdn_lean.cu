@@ -729,8 +729,8 @@ gdn_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         }
         for (int c = 0; c < nchunks; ++c) {
             const float* gates = reinterpret_cast<const float*>(sm + CS_GATES + (c & 3) * 1280);
-            w.wait_hot(CB_V, c & 1);
             if (c > 0) w.wait_hot(CB_O, (c - 1) & 1);     // O2 of the previous chunk no longer reads bf16 v_new
+            w.wait_hot(CB_V, c & 1);
             tc_fence_after_sync();
             if (tid == 0) stamp(0, c, 0);
             {
@@ -764,8 +764,8 @@ gdn_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             tc_fence_before_sync();
             mbar_arrive(w.bar(CB_VREADY));
             if (tid == 0) stamp(0, c, 1);
-            w.wait_hot(CB_S, c & 1);
             w.wait_hot(CB_O1, c & 1);                      // O1 of this chunk no longer reads the bf16 state
+            w.wait_hot(CB_S, c & 1);
             tc_fence_after_sync();
             if (tid == 0) stamp(0, c, 2);
             const float gamma = gates[256];
@@ -861,9 +861,11 @@ gdn_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             for (int c = 0; c < nchunks; ++c) {
                 const uint32_t s = c & 1;
                 const uint64_t dW = dW0 + (uint64_t)((s * STAGE_A) >> 4), dK = dK0 + (uint64_t)((s * STAGE_A) >> 4);
-                w.wait_hot(CB_SREADY, c & 1);
+                // the waits that are normally long satisfied come first: whatever follows the wait on the
+                // state sits on the dependent chain
                 w.wait_hot(CB_FULLA0 + s, (c >> 1) & 1);
                 w.wait_hot(CB_U, c & 1);                       // U^T of this chunk is in the accumulator
+                w.wait_hot(CB_SREADY, c & 1);
                 tc_fence_after_sync();
                 stamp(1, c, 0);
 #pragma unroll
