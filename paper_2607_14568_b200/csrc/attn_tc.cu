@@ -269,14 +269,15 @@ attn_causal_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             for (int j = 0; j < ntiles; ++j) {
                 const uint32_t s = j & 1, s1 = (j + 1) & 1;
                 const bool more = (j + 1 < ntiles);
+                // the tiles are normally there long before the probabilities: these waits come first, so that
+                // nothing but the MMAs sits between "P ready" and "next scores ready"
                 w.wait(AB_VFULL0 + s, (j >> 1) & 1);
+                if (more) w.wait(AB_KFULL0 + s1, ((j + 1) >> 1) & 1);
                 if (j < nA) {
                     w.wait(AB_PFULL0 + 0, j & 1);
                     tc_fence_after_sync();
                     issue_pv(0, j);
                     if (j + 1 < nA) {
-                        w.wait(AB_KFULL0 + s1, ((j + 1) >> 1) & 1);
-                        tc_fence_after_sync();
                         issue_qk(0, j + 1);
                     } else {
                         mma_commit(w.bar(AB_PVDONE0 + 0));
@@ -287,8 +288,6 @@ attn_causal_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                     tc_fence_after_sync();
                     issue_pv(1, j);
                     if (more) {
-                        w.wait(AB_KFULL0 + s1, ((j + 1) >> 1) & 1);
-                        tc_fence_after_sync();
                         issue_qk(1, j + 1);
                     } else {
                         mma_commit(w.bar(AB_PVDONE0 + 1));
