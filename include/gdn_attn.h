@@ -12,6 +12,10 @@
  *
  * Layouts (row-major, DEVICE pointers, 16-byte aligned): q, out [B, T, Hq, d]; k, v [B, T, Hkv, d];
  * bf16 storage, fp32 scores, softmax and accumulation, `out` rounded to nearest even.
+ * With cu_seqlens != NULL (B + 1 ascending int32 on the device, cu_seqlens[0] = 0, cu_seqlens[B] = T)
+ * the tensors are packed [T, H, d] with T the total number of tokens, as in gdn_chunk_prefill:
+ * sequence n owns tokens [cu_seqlens[n], cu_seqlens[n+1]) and attends only to itself; empty
+ * sequences are allowed.
  * Supported: d = 128, Hq a positive multiple of Hkv.  Where the paper writes the score matrix to
  * a buffer (heads x T x T floats), this library keeps 128 x 128 tiles of it in tensor memory only.
  *
@@ -30,6 +34,7 @@ extern "C" {
 #endif
 
 int gdn_attn_causal_prefill(const void* q, const void* k, const void* v, void* out,
+                            const int32_t* cu_seqlens,
                             int B, int T, int Hq, int Hkv, int d, float scale,
                             gdn_stream_t stream);
 

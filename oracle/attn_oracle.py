@@ -11,7 +11,8 @@ heads share one key/value head by addressing the same K/V block.
                        that normalises the valid prefix and writes exact zeros beyond it, full
                        rectangular product with V
 Layouts: q [B,T,Hq,d], k, v [B,T,Hkv,d], out [B,T,Hq,d]; query head h reads key/value head
-h // (Hq // Hkv).  `scale` multiplies the scores (the usual choice is 1/sqrt(d)).  Plain numpy.
+h // (Hq // Hkv).  `scale` multiplies the scores (the usual choice is 1/sqrt(d)).  With cu_seqlens the
+tensors are packed [T,H,d] and every sequence attends to itself only.  Plain numpy.
 """
 from __future__ import annotations
 
@@ -29,8 +30,15 @@ def _check(q, k, v):
         raise ValueError("Hq must be a multiple of Hkv")
 
 
-def attention_causal(q, k, v, scale):
+def attention_causal(q, k, v, scale, cu_seqlens=None):
     q, k, v = _f64(q), _f64(k), _f64(v)
+    if cu_seqlens is not None:          # packed [T,H,d]: every sequence on its own
+        cu = [int(x) for x in np.asarray(cu_seqlens)]
+        out = np.zeros(q.shape[:-1] + (v.shape[-1],))
+        for a, b in zip(cu[:-1], cu[1:]):
+            if b > a:
+                out[a:b] = attention_causal(q[None, a:b], k[None, a:b], v[None, a:b], scale)[0]
+        return out
     _check(q, k, v)
     B, T, Hq, d = q.shape
     group = Hq // k.shape[2]

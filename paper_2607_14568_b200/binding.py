@@ -52,7 +52,7 @@ def lib():
         L.gdn_chunk_prefill_snapshots.restype = i
         L.gdn_chunk_prefill_raw.argtypes = [vp] * 5 + [ctypes.c_float] * 2 + [vp] * 4 + [i] * 6 + [vp]
         L.gdn_chunk_prefill_raw.restype = i
-        L.gdn_attn_causal_prefill.argtypes = [vp] * 4 + [i] * 5 + [ctypes.c_float, vp]
+        L.gdn_attn_causal_prefill.argtypes = [vp] * 5 + [i] * 5 + [ctypes.c_float, vp]
         L.gdn_attn_causal_prefill.restype = i
         L.gdn_workspace_bytes.argtypes = [i] * 6
         L.gdn_workspace_bytes.restype = sz
@@ -251,19 +251,25 @@ def gdn_chunk_prefill_raw(q_raw, k_raw, v, a_raw, b_raw, gate_scale, norm_eps, i
     return out, final_state
 
 
-def gdn_attn_causal_prefill(q, k, v, out, scale=None, stream=None):
-    """Causal softmax attention with grouped queries: q, out [B,T,Hq,d], k, v [B,T,Hkv,d] bf16 on the device;
-    scale defaults to 1/sqrt(d).  See include/gdn_attn.h."""
+def gdn_attn_causal_prefill(q, k, v, out, scale=None, cu_seqlens=None, stream=None):
+    """Causal softmax attention with grouped queries: q, out [B,T,Hq,d], k, v [B,T,Hkv,d] bf16 on the device
+    (packed [T,H,d] with int32 cu_seqlens [B+1]); scale defaults to 1/sqrt(d).  See include/gdn_attn.h."""
     bf = torch.bfloat16
-    _check([("q", q, bf), ("k", k, bf), ("v", v, bf), ("out", out, bf)], bf, "cuda")
-    if q.dim() != 4 or k.dim() != 4 or v.shape != k.shape or out.shape != q.shape or q.shape[:2] != k.shape[:2] \
-            or q.shape[3] != k.shape[3]:
-        raise ValueError("q, out [B,T,Hq,d] and k, v [B,T,Hkv,d] expected")
-    B, T, Hq, d = q.shape
+    _check([("q", q, bf), ("k", k, bf), ("v", v, bf), ("out", out, bf), ("cu_seqlens", cu_seqlens, torch.int32)],
+           bf, "cuda")
+    nd = 4 if cu_seqlens is None else 3
+    if q.dim() != nd or k.dim() != nd or v.shape != k.shape or out.shape != q.shape or q.shape[:-2] != k.shape[:-2] \
+            or q.shape[-1] != k.shape[-1]:
+        raise ValueError("q, out [B,T,Hq,d] and k, v [B,T,Hkv,d] expected (packed: [T,H,d])")
+    if cu_seqlens is None:
+        B, T = q.shape[0], q.shape[1]
+    else:
+        B, T = cu_seqlens.numel() - 1, q.shape[0]
+    Hq, d = q.shape[-2], q.shape[-1]
     if scale is None:
         scale = 1.0 / float(d) ** 0.5
-    rc = lib().gdn_attn_causal_prefill(_ptr(q), _ptr(k), _ptr(v), _ptr(out), int(B), int(T), int(Hq), int(k.shape[2]),
-                                       int(d), float(scale), _stream(stream))
+    rc = lib().gdn_attn_causal_prefill(_ptr(q), _ptr(k), _ptr(v), _ptr(out), _ptr(cu_seqlens), int(B), int(T), int(Hq),
+                                       int(k.shape[-2]), int(d), float(scale), _stream(stream))
     if rc != 0:
         raise GdnError(rc, "gdn_attn_causal_prefill")
     return out

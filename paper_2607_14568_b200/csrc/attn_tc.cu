@@ -77,7 +77,8 @@ struct AWaiter {
 };
 
 struct AttnParams {
-    __nv_bfloat16* out;      // [B, T, Hq, 128]
+    __nv_bfloat16* out;      // [B, T, Hq, 128], or packed [T, Hq, 128]
+    const int32_t* cu;       // packed input: B + 1 sequence boundaries (device), else nullptr
     int B, T, Hq, Hkv;
     float scale_log2e;       // scale * log2(e)
 };
@@ -98,10 +99,26 @@ attn_causal_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
     AWaiter w{base + AS_BARS, reinterpret_cast<volatile int*>(sm + AS_MISC + 4)};
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int nqt = (p.T + BM - 1) / BM;
-    const int npair = (nqt + 1) / 2;
-    const int t = npair - 1 - (int)blockIdx.y;             // CTAs start in x-major order: every head's longest
-    const int h = blockIdx.x, b = blockIdx.z;              // pair of tiles first, the short ones fill the tail
+    // which sequence and which pair of query tiles: batched input takes them from the grid; packed input
+    // walks the sequence boundaries (grid.y covers an upper bound of the pair count, the surplus CTAs leave)
+    int tok0, len, t;
+    if (p.cu) {
+        int y = (int)blockIdx.y, n = 0;
+        tok0 = 0; len = 0; t = -1;
+        for (; n < p.B; ++n) {
+            const int a = p.cu[n], l = p.cu[n + 1] - a;
+            const int np = ((l + BM - 1) / BM + 1) / 2;
+            if (y < np) { tok0 = a; len = l; t = np - 1 - y; break; }
+            y -= np;
+        }
+        if (t < 0) return;                                 // uniform for the CTA; nothing has been set up yet
+    } else {
+        tok0 = (int)blockIdx.z * p.T;
+        len = p.T;
+        t = (((len + BM - 1) / BM + 1) / 2) - 1 - (int)blockIdx.y;   // CTAs start in x-major order: every head's
+    }                                                      // longest pair of tiles first, the short ones fill the tail
+    const int nqt = (len + BM - 1) / BM;
+    const int h = blockIdx.x;
     const int hk = h / (p.Hq / p.Hkv);                     // the key/value head this query head reads
     const bool hasB = (2 * t + 1 < nqt);
     const int nA = 2 * t + 1;                              // key tiles of A: 0..2t (the last is its diagonal)
@@ -218,13 +235,13 @@ attn_causal_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             tc_fence_after_sync();
             const float inv = 1.0f / l;
             const int row = qt * BM + r;
-            __nv_bfloat16* dst = p.out + ((size_t)(b * p.T + row) * p.Hq + h) * HD;
+            __nv_bfloat16* dst = p.out + ((size_t)(tok0 + row) * p.Hq + h) * HD;
 #pragma unroll
             for (int q4 = 0; q4 < 4; ++q4) {
                 uint32_t o[32];
                 tmem_ld32(to + 32 * q4, o);
                 tmem_wait_ld();
-                if (row < p.T) {
+                if (row < len) {
 #pragma unroll
                     for (int cc = 0; cc < 4; ++cc) {
                         uint4 val;
@@ -309,13 +326,13 @@ attn_causal_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                 tma_load_3d(dst + 16384, map, 64, head, tok, full);
                 tma_load_3d(dst + 24576, map, 64, head, tok + 64, full);
             };
-            const int tok_q = b * p.T + 2 * t * BM;
+            const int tok_q = tok0 + 2 * t * BM;
             mbar_arrive_expect_tx(w.bar(AB_Q), hasB ? 2 * TILE_BYTES : TILE_BYTES);
             load_tile(base + AS_Q, &map_q, h, tok_q, w.bar(AB_Q));
             if (hasB) load_tile(base + AS_Q + TILE_BYTES, &map_q, h, tok_q + BM, w.bar(AB_Q));
             for (int j = 0; j < ntiles; ++j) {
                 const uint32_t s = j & 1;
-                const int tok = b * p.T + j * BN;
+                const int tok = tok0 + j * BN;
                 if (j >= 2) w.wait(AB_KFREE0 + s, ((j >> 1) - 1) & 1);
                 mbar_arrive_expect_tx(w.bar(AB_KFULL0 + s), TILE_BYTES);
                 load_tile(base + AS_K + s * TILE_BYTES, &map_k, hk, tok, w.bar(AB_KFULL0 + s));
@@ -353,19 +370,20 @@ int attn_query_status() {
     return st;
 }
 
-int launch_attn(const void* q, const void* k, const void* v, void* out, int B, int T, int Hq, int Hkv, int d,
-                float scale, cudaStream_t stream) {
+int launch_attn(const void* q, const void* k, const void* v, void* out, const int32_t* cu_seqlens, int B, int T,
+                int Hq, int Hkv, int d, float scale, cudaStream_t stream) {
     if (!attn_supported(Hq, Hkv, d)) return GDN_ERR_UNSUPPORTED;
-    if (B > 65535 || ((T + BM - 1) / BM + 1) / 2 > 65535) return GDN_ERR_UNSUPPORTED;
+    if (B > 65535 || T / (2 * BM) + B + 1 > 65535) return GDN_ERR_UNSUPPORTED;
     if (B == 0 || T == 0) return GDN_OK;
-    const uint64_t tokens = (uint64_t)B * T;
+    const uint64_t tokens = cu_seqlens ? (uint64_t)T : (uint64_t)B * T;
     if (tokens > 0x7fffffffull) return GDN_ERR_TOO_LARGE;
     CUtensorMap mq, mk, mv;
     if (!tc_make_map(&mq, q, tokens, Hq, d) || !tc_make_map(&mk, k, tokens, Hkv, d) ||
         !tc_make_map(&mv, v, tokens, Hkv, d))
         return GDN_ERR_CUDA;
-    AttnParams p{static_cast<__nv_bfloat16*>(out), B, T, Hq, Hkv, scale * 1.4426950408889634f};
-    dim3 grid(Hq, ((T + BM - 1) / BM + 1) / 2, B);
+    AttnParams p{static_cast<__nv_bfloat16*>(out), cu_seqlens, B, T, Hq, Hkv, scale * 1.4426950408889634f};
+    // packed: sum over sequences of ceil(ceil(len / 128) / 2) <= T / 256 + B
+    dim3 grid(Hq, cu_seqlens ? T / (2 * BM) + B : ((T + BM - 1) / BM + 1) / 2, cu_seqlens ? 1 : B);
     if (cudaFuncSetAttribute(attn_causal_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ATTN_SMEM) !=
         cudaSuccess)
         return GDN_ERR_CUDA;

@@ -237,13 +237,13 @@ int gdn_set_workspace(void* device_ptr, size_t bytes) {
     return GDN_OK;
 }
 
-int gdn_attn_causal_prefill(const void* q, const void* k, const void* v, void* out, int B, int T, int Hq, int Hkv,
-                            int d, float scale, gdn_stream_t stream) {
+int gdn_attn_causal_prefill(const void* q, const void* k, const void* v, void* out, const int32_t* cu_seqlens,
+                            int B, int T, int Hq, int Hkv, int d, float scale, gdn_stream_t stream) {
     if (B < 0 || T < 0 || Hq <= 0 || Hkv <= 0 || d <= 0 || !(scale >= 0.f) || scale - scale != 0.f)
         return GDN_ERR_INVALID_ARG;
     if ((B > 0 && T > 0) && (!q || !k || !v || !out)) return GDN_ERR_INVALID_ARG;
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out)) return GDN_ERR_UNSUPPORTED;
-    return launch_attn(q, k, v, out, B, T, Hq, Hkv, d, scale, reinterpret_cast<cudaStream_t>(stream));
+    return launch_attn(q, k, v, out, cu_seqlens, B, T, Hq, Hkv, d, scale, reinterpret_cast<cudaStream_t>(stream));
 }
 
 int gdn_query_status(void) {

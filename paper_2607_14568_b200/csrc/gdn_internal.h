@@ -67,8 +67,8 @@ int launch_decode(const void* q, const void* k, const void* v, const float* log_
 
 // Causal grouped-query softmax attention (bf16, d = 128).
 bool attn_supported(int Hq, int Hkv, int d);
-int launch_attn(const void* q, const void* k, const void* v, void* out, int B, int T, int Hq, int Hkv, int d,
-                float scale, cudaStream_t stream);
+int launch_attn(const void* q, const void* k, const void* v, void* out, const int32_t* cu_seqlens, int B, int T,
+                int Hq, int Hkv, int d, float scale, cudaStream_t stream);
 int attn_query_status();
 
 void count_launch(int n = 1);

@@ -94,3 +94,14 @@ def test_product_softmax_product_form_equals_the_definition():
     qt, kt, vt = (torch.from_numpy(x).permute(0, 2, 1, 3) for x in (q, np.repeat(k, 2, axis=2), np.repeat(v, 2, axis=2)))
     ref = torch.nn.functional.scaled_dot_product_attention(qt, kt, vt, is_causal=True, scale=0.25)
     np.testing.assert_allclose(a, ref.permute(0, 2, 1, 3).numpy(), rtol=1e-10, atol=1e-12)
+
+
+def test_packed_sequences_are_independent():
+    rng = np.random.default_rng(4)
+    q, k, v = _rand(rng, B=1, T=20, Hq=2, Hkv=1, d=4)
+    cu = [0, 7, 7, 20]
+    packed = oracle.attention_causal(q[0], k[0], v[0], 0.4, cu_seqlens=cu)
+    np.testing.assert_allclose(packed[:7], oracle.attention_causal(q[:, :7], k[:, :7], v[:, :7], 0.4)[0], rtol=1e-14)
+    np.testing.assert_allclose(packed[7:], oracle.attention_causal(q[:, 7:], k[:, 7:], v[:, 7:], 0.4)[0], rtol=1e-14)
+    # first token of every sequence returns its own value: nothing leaks across the boundary
+    np.testing.assert_allclose(packed[7, 0], v[0, 7, 0], rtol=1e-14)

@@ -95,3 +95,19 @@ def test_errors():
     with pytest.raises(gdn.GdnError) as e:
         gdn.gdn_attn_causal_prefill(q64, q64, q64, torch.empty_like(q64))  # d = 64
     assert e.value.status == 2
+
+
+def test_packed_sequences():
+    """Packed input: ragged lengths, an empty sequence, a one-token sequence; no leakage between sequences."""
+    import paper_2607_14568_b200 as gdn
+    lengths = [300, 0, 1, 129, 512, 77]
+    cu = np.concatenate([[0], np.cumsum(lengths)]).astype(np.int32)
+    cfg = get_attn_config("attn_small", B=1, T=int(cu[-1]), Hq=4, Hkv=2)
+    q, k, v = (a[0] for a in make_attn_inputs(cfg))          # [T, H, d]
+    dq, dk, dv = _dev(q), _dev(k), _dev(v)
+    out = torch.full_like(dq, float("nan"))
+    gdn.gdn_attn_causal_prefill(dq, dk, dv, out, cfg.scale, cu_seqlens=torch.from_numpy(cu).cuda())
+    torch.cuda.synchronize()
+    assert gdn.gdn_query_status() == 0
+    want = oracle.attention_causal(widen(q), widen(k), widen(v), cfg.scale, cu_seqlens=cu)
+    assert_close(f64(out), want, ATTN_REL_L2, ATTN_MAX_ABS, "out")
