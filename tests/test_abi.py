@@ -62,3 +62,36 @@ def test_host_entry_rejects_bad_arguments_without_a_gpu(libpath):
     rc = lib.gdn_chunk_prefill_host(p, p, p, p, p, None, p, None, cu.ctypes.data_as(vp), 1, 64, 1, 128, 128, 64,
                                     vp(256), ctypes.c_size_t(1 << 30), None)
     assert rc == 1   # cu_seqlens[B] != T
+
+
+def test_widened_entry_points_reject_bad_arguments_without_a_gpu(libpath):
+    """The argument checks of the attention, snapshot and raw-projection entry points come before any
+    CUDA call, so they can be exercised on a machine without a GPU (pointers are never dereferenced)."""
+    lib = ctypes.CDLL(libpath)
+    vp, f = ctypes.c_void_p, ctypes.c_float
+    p = vp(4096)                                                    # aligned, never dereferenced
+    attn = lib.gdn_attn_causal_prefill
+    attn.restype = ctypes.c_int
+    attn.argtypes = [vp] * 5 + [ctypes.c_int] * 5 + [f, vp]
+    assert attn(p, p, p, p, None, -1, 64, 2, 1, 128, 0.1, None) == 1       # negative B
+    assert attn(p, p, p, p, None, 1, 64, 2, 1, 128, -0.1, None) == 1       # negative scale
+    assert attn(p, p, p, p, None, 1, 64, 2, 1, 128, float("nan"), None) == 1
+    assert attn(None, p, p, p, None, 1, 64, 2, 1, 128, 0.1, None) == 1     # null q
+    assert attn(vp(4100), p, p, p, None, 1, 64, 2, 1, 128, 0.1, None) == 2  # misaligned
+    assert attn(p, p, p, p, None, 1, 64, 3, 2, 128, 0.1, None) == 2        # 3 query heads on 2 kv heads
+    assert attn(p, p, p, p, None, 1, 64, 2, 1, 64, 0.1, None) == 2         # d = 64
+    assert attn(p, p, p, p, None, 0, 64, 2, 1, 128, 0.1, None) == 0        # empty batch: nothing to do
+    raw = lib.gdn_chunk_prefill_raw
+    raw.restype = ctypes.c_int
+    raw.argtypes = [vp] * 5 + [f, f] + [vp] * 4 + [ctypes.c_int] * 6 + [vp]
+    assert raw(p, p, p, p, p, -1.0, 0.0, None, p, None, None, 1, 64, 1, 128, 128, 64, None) == 1   # negative gate scale
+    assert raw(p, p, p, p, p, 0.05, -1.0, None, p, None, None, 1, 64, 1, 128, 128, 64, None) == 1  # negative eps
+    assert raw(p, p, p, p, p, 0.05, 0.0, None, p, None, None, 1, 64, 1, 128, 128, 32, None) == 2   # chunk != 64
+    assert raw(p, p, p, p, p, 0.05, 0.0, None, p, None, None, 1, 64, 1, 64, 64, 64, None) == 2     # d = 64
+    assert raw(p, p, p, p, p, 0.05, 0.0, None, p, None, None, 1, 64, 1, 128, 128, 64, None) == 3   # no workspace set
+    snap = lib.gdn_chunk_prefill_snapshots
+    snap.restype = ctypes.c_int
+    snap.argtypes = [vp] * 8 + [ctypes.c_int] * 7 + [vp, vp]
+    assert snap(p, p, p, p, p, None, p, None, 1, 128, 1, 128, 128, 64, 0, p, None) == 1            # every 0 chunks
+    assert snap(p, p, p, p, p, None, p, None, 1, 128, 1, 128, 128, 64, 1, None, None) == 1         # no snapshot buffer
+    assert snap(p, p, p, p, p, None, p, None, 1, 128, 1, 128, 128, 64, 1, p, None) == 3            # no workspace set
