@@ -1,6 +1,6 @@
 // Thin inline-PTX wrappers for sm_100a: mbarrier, TMA (cp.async.bulk.tensor), tensor
 // memory (tcgen05.alloc/ld/st) and the 5th-generation tensor core (tcgen05.mma).
-// No cluster multicast is used anywhere.
+// Every copy is issued by one CTA for itself.
 #pragma once
 
 #include <cuda.h>
@@ -66,7 +66,7 @@ __device__ __forceinline__ void named_bar_sync(uint32_t id, uint32_t nthreads) {
     asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
 }
 
-// ---------------------------------------------------------------- TMA (tiled, 3-D, no multicast)
+// ---------------------------------------------------------------- TMA (tiled, 3-D, one CTA)
 __device__ __forceinline__ void tma_load_3d(uint32_t smem_dst, const CUtensorMap* map, int c0, int c1, int c2,
                                             uint32_t bar) {
     asm volatile(
