@@ -204,6 +204,7 @@ gdn_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int H = p.H;
+    pdl_trigger();                      // the next kernel of the call may set itself up while this one runs
     if (tid == 0) {
         mbar_init(w.bar(PB_FULL), 1); mbar_init(w.bar(PB_G), 1); mbar_init(w.bar(PB_W), 1);
         mbar_init(w.bar(PB_TREADY), 128); mbar_init(w.bar(PB_GREADY), 32); mbar_init(w.bar(PB_DONE), 128);
@@ -693,6 +694,7 @@ gdn_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem = sMisc[0];
+    pdl_wait();                         // scratch items and incoming states come from the kernels before this one
     const unsigned long long t_start = DBG ? globaltimer_ns() : 0ull;
     auto stamp = [&](int role, int c, int ev) {
         if (DBG && p.dbg && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && c < 32)
@@ -1049,6 +1051,8 @@ gdn_summary_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem = sMisc[0];
+    pdl_trigger();
+    pdl_wait();                         // the scratch items come from the prepare kernel
 
     if (warp < 8) {
         // ======================= two chain warpgroups: values (0) and identity (1) =======================
@@ -1247,6 +1251,8 @@ __global__ void __launch_bounds__(CMB_THREADS) gdn_combine_kernel(CombineParams 
         const int i = idx / CMB_COLS, j = idx % CMB_COLS;
         sS[i][j] = p.s0 ? p.s0[(((size_t)n * H + h) * DK + i) * dv + j0 + j] : 0.f;
     }
+    pdl_trigger();
+    pdl_wait();                         // M_seg, N_seg come from the summary kernel (the initial state loaded above is an input)
     __syncthreads();
     if (tid == 0)
         for (int sg = 0; sg < (int)CMB_BUFS && sg + 1 < p.nseg; ++sg) load_mt(sg);
@@ -1326,6 +1332,22 @@ int lean_init_workspace(void* workspace) {
     return cudaMemset(workspace, 0, kWorkspaceHeader) == cudaSuccess ? GDN_OK : GDN_ERR_CUDA;
 }
 
+// Launch a kernel that may begin (set-up only, up to its pdl_wait) before the previous kernel in the stream ends.
+template <typename... KArgs, typename... Args>
+static void launch_after(void (*kernel)(KArgs...), dim3 grid, int threads, size_t smem, cudaStream_t stream, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = dim3(threads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = g_lean_timing ? 0 : 1;   // events between kernels: plain order
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
 size_t lean_workspace_bytes(int B, int T, int H, int d_k, int d_v, bool packed) {
     if (!tc_supported(d_k, d_v) || B <= 0 || T < 0 || H <= 0) return 0;
     const size_t tokens = packed ? (size_t)T : (size_t)B * T;
@@ -1402,13 +1424,13 @@ int launch_lean(const PrefillArgs& a, void* workspace, size_t workspace_bytes, c
         float* seg_mt = seg_n + state_elems;
         SummaryParams sp{a.cu_seqlens, ws, seg_n, seg_mt, a.B, a.T, a.H, a.d_v, nseg, seg_chunks};
         dim3 sgrid(a.d_v / DVB, a.H, a.B * (nseg - 1));
-        gdn_summary_kernel<<<sgrid, SUM_THREADS, SUM_SMEM, stream>>>(mk, mv, sp);
+        launch_after(gdn_summary_kernel, sgrid, SUM_THREADS, SUM_SMEM, stream, mk, mv, sp);
         count_launch();
         if (cudaGetLastError() != cudaSuccess) return GDN_ERR_CUDA;
         mark(2);
         CombineParams cb{a.initial_state, seg_n, seg_mt, seg_sin, a.H, a.d_v, nseg};
         dim3 cgrid(a.d_v / CMB_COLS, a.H, a.B);
-        gdn_combine_kernel<<<cgrid, CMB_THREADS, CMB_SMEM, stream>>>(cb);
+        launch_after(gdn_combine_kernel, cgrid, CMB_THREADS, CMB_SMEM, stream, cb);
         count_launch();
         if (cudaGetLastError() != cudaSuccess) return GDN_ERR_CUDA;
         mark(3);
@@ -1419,8 +1441,8 @@ int launch_lean(const PrefillArgs& a, void* workspace, size_t workspace_bytes, c
                    ws, seg_sin, g_lean_dbg, g_lean_drop_chunk, a.B, a.T, a.H, a.d_v, nseg, seg_chunks,
                    snaps, snap_every, snaps ? (a.T / C) / snap_every : 0};
     dim3 grid(a.d_v / DVB, a.H, a.B * nseg);
-    if (g_lean_dbg) gdn_chain_kernel<true><<<grid, CHAIN_THREADS, CHAIN_SMEM, stream>>>(mq, mk, mv, cp);
-    else gdn_chain_kernel<false><<<grid, CHAIN_THREADS, CHAIN_SMEM, stream>>>(mq, mk, mv, cp);
+    if (g_lean_dbg) launch_after(gdn_chain_kernel<true>, grid, CHAIN_THREADS, CHAIN_SMEM, stream, mq, mk, mv, cp);
+    else launch_after(gdn_chain_kernel<false>, grid, CHAIN_THREADS, CHAIN_SMEM, stream, mq, mk, mv, cp);
     count_launch();
     mark(4);
     return cudaGetLastError() == cudaSuccess ? GDN_OK : GDN_ERR_CUDA;
