@@ -68,6 +68,9 @@ typedef struct CUstream_st* gdn_stream_t;
  * chunked delta-rule scan for the recurrent layers").  Supported: chunk = 64,
  * d_k = 128, d_v a multiple of 128 (tensor-core path); other d_k, d_v that are
  * multiples of 32 with d_k <= 128 fall back to the fp32-arithmetic kernel below.
+ * The call makes no host-device copy and no synchronisation, so it can be
+ * recorded into a CUDA graph and replayed on new contents of the same buffers
+ * (set the workspace before the capture: gdn_set_workspace synchronises).
  */
 int gdn_chunk_prefill(const void* q, const void* k, const void* v,
                       const float* log_alpha, const float* beta,
