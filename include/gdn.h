@@ -114,6 +114,11 @@ int gdn_chunk_prefill_bf16_simt(const void* q, const void* k, const void* v,
  * without synchronising.  staging_dev is caller-owned device memory of at least
  * gdn_host_staging_bytes(...) bytes, 256-byte aligned.  cu_seqlens_host may be
  * NULL; initial_state_host / final_state_host may be NULL as above.
+ * One long sequence (B = 1, no cu_seqlens, T >= 4096, d_k = 128) is processed in
+ * pieces of 2048 tokens with the fp32 state carried from piece to piece: uploads,
+ * kernels and downloads of different pieces overlap on two copy streams that the
+ * library creates once (with their events; nothing else is ever allocated).  The
+ * call is still complete on `stream` when everything has reached the host.
  * Errors: as gdn_chunk_prefill, plus GDN_ERR_WORKSPACE when staging is too small.
  */
 int gdn_chunk_prefill_host(const void* q_host, const void* k_host, const void* v_host,

@@ -1,6 +1,7 @@
 // C-ABI entry points of libgdn: argument validation and dispatch.  See include/gdn.h.
 
 #include <atomic>
+#include <vector>
 
 #include "gdn_internal.h"
 #include "gdn_attn.h"
@@ -77,6 +78,74 @@ bool staging_layout(int B, int T, int H, int d_k, int d_v, bool packed, Staging*
     return true;
 }
 
+// One long sequence through the host-buffer entry point: the sequence is cut into pieces of kHostPiece
+// tokens whose upload, prefill (the state carried from piece to piece, exactly, in fp32) and download run
+// on three streams, so that the two PCIe directions and the kernels overlap instead of following each other.
+constexpr int kHostPiece = 2048;
+
+struct HostPipe {
+    cudaStream_t s_in = nullptr, s_out = nullptr;
+    std::vector<cudaEvent_t> ev;
+    bool ensure(size_t n) {
+        if (!s_in && cudaStreamCreateWithFlags(&s_in, cudaStreamNonBlocking) != cudaSuccess) return false;
+        if (!s_out && cudaStreamCreateWithFlags(&s_out, cudaStreamNonBlocking) != cudaSuccess) return false;
+        while (ev.size() < n) {
+            cudaEvent_t e;
+            if (cudaEventCreateWithFlags(&e, cudaEventDisableTiming) != cudaSuccess) return false;
+            ev.push_back(e);
+        }
+        return true;
+    }
+};
+HostPipe g_host_pipe;
+
+int host_pipelined(const void* q_host, const void* k_host, const void* v_host, const float* a_host, const float* b_host,
+                   const float* s0_host, void* out_host, float* sT_host, int T, int H, int d_k, int d_v, char* base,
+                   const Staging& L, cudaStream_t stream) {
+    const int npieces = (T + kHostPiece - 1) / kHostPiece;
+    HostPipe& hp = g_host_pipe;
+    if (!hp.ensure(2 * (size_t)npieces + 2)) return GDN_ERR_CUDA;
+    auto ok = [](cudaError_t e) { return e == cudaSuccess; };
+    cudaEvent_t ev_start = hp.ev[0], ev_done = hp.ev[1];
+    // the copy streams start after whatever the caller has already queued on `stream`
+    if (!ok(cudaEventRecord(ev_start, stream)) || !ok(cudaStreamWaitEvent(hp.s_in, ev_start, 0)) ||
+        !ok(cudaStreamWaitEvent(hp.s_out, ev_start, 0)))
+        return GDN_ERR_CUDA;
+    if (s0_host && !ok(cudaMemcpyAsync(base + L.s0, s0_host, L.n_state, cudaMemcpyHostToDevice, hp.s_in)))
+        return GDN_ERR_CUDA;
+    float* carry = reinterpret_cast<float*>(base + L.sT);           // the state between pieces, and the final state
+    const size_t row_qk = (size_t)H * d_k * sizeof(__nv_bfloat16), row_v = (size_t)H * d_v * sizeof(__nv_bfloat16);
+    const size_t row_g = (size_t)H * sizeof(float);
+    for (int p = 0; p < npieces; ++p) {
+        const size_t t0 = (size_t)p * kHostPiece;
+        const int tl = (int)((size_t)T - t0 < (size_t)kHostPiece ? (size_t)T - t0 : (size_t)kHostPiece);
+        auto up = [&](size_t off, const void* src, size_t row) {
+            return ok(cudaMemcpyAsync(base + off + t0 * row, static_cast<const char*>(src) + t0 * row, (size_t)tl * row,
+                                      cudaMemcpyHostToDevice, hp.s_in));
+        };
+        if (!up(L.q, q_host, row_qk) || !up(L.k, k_host, row_qk) || !up(L.v, v_host, row_v) ||
+            !up(L.a, a_host, row_g) || !up(L.b, b_host, row_g))
+            return GDN_ERR_CUDA;
+        cudaEvent_t ev_in = hp.ev[2 + 2 * p], ev_c = hp.ev[3 + 2 * p];
+        if (!ok(cudaEventRecord(ev_in, hp.s_in)) || !ok(cudaStreamWaitEvent(stream, ev_in, 0))) return GDN_ERR_CUDA;
+        const float* s_in = p == 0 ? (s0_host ? reinterpret_cast<const float*>(base + L.s0) : nullptr) : carry;
+        const PrefillArgs a = pack(base + L.q + t0 * row_qk, base + L.k + t0 * row_qk, base + L.v + t0 * row_v,
+                                   reinterpret_cast<const float*>(base + L.a + t0 * row_g),
+                                   reinterpret_cast<const float*>(base + L.b + t0 * row_g), s_in,
+                                   base + L.out + t0 * row_v, carry, nullptr, 1, tl, H, d_k, d_v);
+        if (int rc = validate(a, kChunk)) return rc;
+        if (int rc = dispatch_bf16(a, stream)) return rc;
+        if (!ok(cudaEventRecord(ev_c, stream)) || !ok(cudaStreamWaitEvent(hp.s_out, ev_c, 0)) ||
+            !ok(cudaMemcpyAsync(static_cast<char*>(out_host) + t0 * row_v, base + L.out + t0 * row_v, (size_t)tl * row_v,
+                                cudaMemcpyDeviceToHost, hp.s_out)))
+            return GDN_ERR_CUDA;
+    }
+    if (sT_host && !ok(cudaMemcpyAsync(sT_host, carry, L.n_state, cudaMemcpyDeviceToHost, hp.s_out))) return GDN_ERR_CUDA;
+    // the call is complete on `stream` when the last download is
+    if (!ok(cudaEventRecord(ev_done, hp.s_out)) || !ok(cudaStreamWaitEvent(stream, ev_done, 0))) return GDN_ERR_CUDA;
+    return GDN_OK;
+}
+
 }  // namespace
 }  // namespace gdn
 
@@ -137,6 +206,9 @@ int gdn_chunk_prefill_host(const void* q_host, const void* k_host, const void* v
     }
     cudaStream_t stream = reinterpret_cast<cudaStream_t>(stream_);
     char* base = static_cast<char*>(staging_dev);
+    if (B == 1 && !cu_seqlens_host && T >= 2 * kHostPiece && tc_supported(d_k, d_v))
+        return host_pipelined(q_host, k_host, v_host, log_alpha_host, beta_host, initial_state_host, out_host,
+                              final_state_host, T, H, d_k, d_v, base, L, stream);
     auto h2d = [&](size_t off, const void* src, size_t bytes) {
         return bytes == 0 || cudaMemcpyAsync(base + off, src, bytes, cudaMemcpyHostToDevice, stream) == cudaSuccess;
     };

@@ -212,6 +212,39 @@ def test_host_entry_matches_device_entry():
     assert e.value.status == 3
 
 
+@pytest.mark.parametrize("with_ws", [False, True])
+def test_host_entry_long_sequence_is_pipelined_in_pieces(with_ws):
+    """One long sequence goes through the host entry point in pieces of 2048 tokens with the state carried
+    between them; the result must still be the recurrence over the whole sequence (ragged last piece, given
+    initial state, final state returned), and two calls in a row must agree."""
+    cfg = get_config("long", T=2048 * 2 + 777, H=2, seed=52)
+    x = make_inputs(cfg)
+    h = to_device(x, device="cpu")
+    h = {k: (v.pin_memory() if v is not None else None) for k, v in h.items()}
+    staging = torch.empty(gdn.gdn_host_staging_bytes(cfg.B, x.T_arg, cfg.H, cfg.d_k, cfg.d_v), dtype=torch.uint8,
+                          device="cuda")
+    ws = None
+    if with_ws:
+        ws = torch.empty(gdn.gdn_workspace_bytes(cfg.B, x.T_arg, cfg.H, cfg.d_k, cfg.d_v, False), dtype=torch.uint8,
+                         device="cuda")
+        gdn.gdn_set_workspace(ws)
+    try:
+        o1, f1 = gdn.gdn_chunk_prefill_host(h["q"], h["k"], h["v"], h["log_alpha"], h["beta"], h["initial_state"],
+                                            h["out"], h["final_state"], None, staging)
+        torch.cuda.synchronize()
+        o1, f1 = o1.clone(), f1.clone()
+        o2, f2 = gdn.gdn_chunk_prefill_host(h["q"], h["k"], h["v"], h["log_alpha"], h["beta"], h["initial_state"],
+                                            h["out"], h["final_state"], None, staging)
+        torch.cuda.synchronize()
+        assert gdn.gdn_query_status() == 0
+    finally:
+        gdn.gdn_set_workspace(None)
+    assert torch.equal(o1, o2) and torch.equal(f1, f2)
+    want_out, want_fin = run_oracle(x)
+    assert_close(f64(o1), want_out, BF16_REL_L2, BF16_MAX_ABS, "out")
+    assert_close(f64(f1), want_fin, BF16_REL_L2, None, "final_state")
+
+
 # ---- error behaviour ---------------------------------------------------------------------------------
 def test_error_codes():
     x = make_inputs(get_config("long", T=64, H=1))
