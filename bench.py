@@ -311,8 +311,8 @@ def run_ours(args):
     kernels = None
     if ws_bytes and gdn.lib().gdn_debug_set_timing(1) == 0:
         import ctypes
-        acc = np.zeros(4)
-        buf = (ctypes.c_float * 4)()
+        acc = np.zeros(5)
+        buf = (ctypes.c_float * 5)()
         for i in range(args.steps):
             flush.fill_(i & 0xFF)
             step()
@@ -321,8 +321,8 @@ def run_ours(args):
         gdn.lib().gdn_debug_set_timing(0)
         tot = float(acc.sum())
         if tot > 0:
-            kernels = {n: {"ms": float(a) / args.steps, "share": float(a) / tot}
-                       for n, a in zip(("gdn_prep_kernel", "gdn_summary_kernel", "gdn_combine_kernel", "gdn_chain_kernel"), acc)}
+            names = ("gdn_prep_kernel", "gdn_summary_kernel", "gdn_combine_kernel", "gdn_chain_kernel", "gdn_scan_kernel")
+            kernels = {n: {"ms": float(a) / args.steps, "share": float(a) / tot} for n, a in zip(names, acc) if a > 0}
 
     # ---- aggregate over ranks: max time, summed tokens ----
     (total_ms, e2e_max), tokens_job = aggregate_over_ranks([total_ms, e2e_ms or 0.0], work["tokens"], args.steps,

@@ -70,6 +70,8 @@ def lib():
         L.gdn_debug_get_timing.restype = i
         L.gdn_debug_force_segments.argtypes = [i]
         L.gdn_debug_force_segments.restype = None
+        L.gdn_debug_set_scan.argtypes = [i]
+        L.gdn_debug_set_scan.restype = None
         L.gdn_query_status.argtypes = []
         L.gdn_query_status.restype = i
         L.gdn_debug_set_dump.argtypes = [vp]

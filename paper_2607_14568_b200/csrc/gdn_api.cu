@@ -301,7 +301,7 @@ int gdn_set_workspace(void* device_ptr, size_t bytes) {
     if (device_ptr && (reinterpret_cast<uintptr_t>(device_ptr) & 255u)) return GDN_ERR_UNSUPPORTED;
     g_workspace = nullptr;
     g_workspace_bytes = 0;
-    if (device_ptr && bytes >= 256) {
+    if (device_ptr && bytes >= 4096) {
         if (int rc = lean_init_workspace(device_ptr)) return rc;
         g_workspace = device_ptr;
         g_workspace_bytes = bytes;
@@ -334,10 +334,12 @@ int gdn_debug_reset_status(void) { return lean_reset_status(); }
 
 // Not part of the public header: per-kernel event timing of the two-kernel pipeline (benchmark).
 int gdn_debug_set_timing(int enable) { return lean_set_timing(enable); }
-int gdn_debug_get_timing(float* ms4) { return ms4 ? lean_get_timing(ms4) : GDN_ERR_INVALID_ARG; }
+int gdn_debug_get_timing(float* ms5) { return ms5 ? lean_get_timing(ms5) : GDN_ERR_INVALID_ARG; }
 
-// Not part of the public header: forces the number of sequence segments (0 = automatic).
+// Not part of the public header: forces the number of sequence segments (0 = automatic); chooses between the
+// merged scan kernel (1, default: used whenever its grid fits the GPU at once) and the three stand-alone kernels (0).
 void gdn_debug_force_segments(int nseg) { lean_force_segments(nseg); }
+void gdn_debug_set_scan(int enable) { lean_set_scan(enable); }
 
 // Not part of the public header: lets the tests capture per-stage intermediates.
 void gdn_debug_set_dump(float* device_buffer) { tc_set_debug_dump(device_buffer); }

@@ -58,7 +58,8 @@ void lean_set_drop_chunk(int c);      // tests only: make one TMA load never hap
 int lean_reset_status();              // tests only: clear the status word
 void lean_set_debug(float* p);        // tests only: time stamps of the chain kernel
 int lean_set_timing(int enable);      // benchmark only: record events around each kernel
-int lean_get_timing(float* ms4);      // {prepare, summary, combine, chain} of the last call
+int lean_get_timing(float* ms5);      // {prepare, summary, combine, chain, scan} of the last call
+void lean_set_scan(int enable);       // tests only: 0 = never merge summary, combine and chain into one launch
 
 // Single-token decode step (bf16 q/k/v/out, fp32 state updated in place).
 bool decode_supported(int d_k, int d_v);

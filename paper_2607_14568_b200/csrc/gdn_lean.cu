@@ -25,6 +25,8 @@
 
 #include <cuda.h>
 
+#include <mutex>
+
 #include "gdn_internal.h"
 #include "sm100_ptx.cuh"
 
@@ -39,6 +41,8 @@ static cudaEvent_t g_lean_events[5] = {nullptr, nullptr, nullptr, nullptr, nullp
 static bool g_lean_split_last = false;
 static float* g_lean_dbg = nullptr;        // debug: time stamps of the chain kernel
 static int g_lean_drop_chunk = -1;         // tests: chunk the chain kernel's TMA thread skips (-1 = none)
+static bool g_lean_use_scan = true;        // tests: false = always the stand-alone summary / combine / chain kernels
+static bool g_lean_scan_last = false;
 
 namespace {
 
@@ -101,6 +105,18 @@ __device__ __forceinline__ void st_shared_f4(uint32_t addr, float a, float b, fl
 __device__ __forceinline__ void st_global_v4(void* p, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
     *reinterpret_cast<uint4*>(p) = make_uint4(a, b, c, d);
 }
+// warp-level TF32 MMA on register fragments: D (16 x 8, fp32) += A (16 x 8) * B (8 x 8)
+__device__ __forceinline__ uint32_t tf32_rna(float x) {
+    uint32_t y;
+    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ void mma_tf32(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+
 // plain (untiled) bulk copy global -> shared; both addresses 16-byte aligned, size % 16 == 0
 __device__ __forceinline__ void bulk_load(uint32_t smem_dst, const void* gsrc, uint32_t bytes, uint32_t bar) {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
@@ -370,95 +386,85 @@ gdn_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                 named_bar_sync(1, 128);
             }
             named_bar_sync(1, 128);
-            // The merges are small fp32 products out of shared memory.  A warp owns 8 rows and a lane one
-            // column: the row operand is read with warp-uniform 16-byte loads (one wavefront each) and
-            // the column operand with one 4-byte load per lane -- shared-memory wavefronts, not FMAs,
-            // bound this kernel.
-            {   // level 1: 16-blocks (1,0) and (3,2):  T21 = -T22 (A21 T11); lanes 16..31 take the second half of i
-                const int pr = warp >> 1, r0 = 8 * (warp & 1), c = lane & 15, ih = lane >> 4;
-                const int lo = 32 * pr, hi = lo + 16;
-                float acc[8];
+            // The merges T21 = -T22 A21 T11 are small dense products: they run as warp-level TF32 MMAs
+            // (m16n8k8, fp32 accumulation) on fragments loaded straight from the fp32 matrix in shared memory.
+            // The left product Z = T22 A21 stays in registers: an accumulator fragment holds columns 2t, 2t+1
+            // of its row, which is what the next MMA wants as its A operand once the contraction index is
+            // renumbered (position t <-> column 2t, position t+4 <-> column 2t+1) on both operands alike.
+            // T (rounded to bf16 afterwards) keeps 11 significant bits through these products.
+            {
+                const int g = lane >> 2, t = lane & 3;
+                if (warp < 2) {   // level 1: the 16-blocks (1,0) and (3,2), one warp each
+                    const int lo = 32 * warp, hi = lo + 16;
+                    float z[2][4] = {};
 #pragma unroll
-                for (int x = 0; x < 8; ++x) acc[x] = 0.f;
+                    for (int ks = 0; ks < 2; ++ks) {
+                        const float2 a01 = *reinterpret_cast<const float2*>(sTf + (hi + g) * LDA + hi + 8 * ks + 2 * t);
+                        const float2 a23 = *reinterpret_cast<const float2*>(sTf + (hi + g + 8) * LDA + hi + 8 * ks + 2 * t);
+                        const uint32_t af[4] = {tf32_rna(a01.x), tf32_rna(a23.x), tf32_rna(a01.y), tf32_rna(a23.y)};
 #pragma unroll
-                for (int i4 = 0; i4 < 2; ++i4) {
-                    const int ib = 8 * ih + 4 * i4;
-                    float tv[4];
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) tv[e] = sTf[(lo + ib + e) * LDA + lo + c];
-#pragma unroll
-                    for (int x = 0; x < 8; ++x) {
-                        const float4 a4 = *reinterpret_cast<const float4*>(sA + (hi + r0 + x) * LDA + lo + ib);
-                        acc[x] = fmaf(a4.x, tv[0], fmaf(a4.y, tv[1], fmaf(a4.z, tv[2], fmaf(a4.w, tv[3], acc[x]))));
+                        for (int q = 0; q < 2; ++q) {
+                            const uint32_t b0 = tf32_rna(sA[(hi + 8 * ks + 2 * t) * LDA + lo + 8 * q + g]);
+                            const uint32_t b1 = tf32_rna(sA[(hi + 8 * ks + 2 * t + 1) * LDA + lo + 8 * q + g]);
+                            mma_tf32(z[q], af, b0, b1);
+                        }
                     }
-                }
+                    float r[2][4] = {};
 #pragma unroll
-                for (int x = 0; x < 8; ++x) {
-                    acc[x] += __shfl_xor_sync(0xffffffffu, acc[x], 16);
-                    if (ih == 0) sY[(16 * pr + r0 + x) * LDY + c] = acc[x];
+                    for (int ks = 0; ks < 2; ++ks) {
+                        const uint32_t af[4] = {tf32_rna(z[ks][0]), tf32_rna(z[ks][2]), tf32_rna(z[ks][1]), tf32_rna(z[ks][3])};
+#pragma unroll
+                        for (int q = 0; q < 2; ++q) {
+                            const uint32_t b0 = tf32_rna(sTf[(lo + 8 * ks + 2 * t) * LDA + lo + 8 * q + g]);
+                            const uint32_t b1 = tf32_rna(sTf[(lo + 8 * ks + 2 * t + 1) * LDA + lo + 8 * q + g]);
+                            mma_tf32(r[q], af, b0, b1);
+                        }
+                    }
+#pragma unroll
+                    for (int q = 0; q < 2; ++q) {      // only this warp reads or writes this block
+                        *reinterpret_cast<float2*>(sTf + (hi + g) * LDA + lo + 8 * q + 2 * t) = make_float2(-r[q][0], -r[q][1]);
+                        *reinterpret_cast<float2*>(sTf + (hi + g + 8) * LDA + lo + 8 * q + 2 * t) = make_float2(-r[q][2], -r[q][3]);
+                    }
                 }
                 named_bar_sync(1, 128);
+                // level 2: the 32-block (1,0); warp = (16 rows mb, 16 columns nb) of the result.  The triangular
+                // factors shorten the contractions: row block 0 of T22 ends at column 16, column block 1 of
+                // T11 starts at row 16.
+                const int mb = warp & 1, nb = warp >> 1;
+                float z[4][4] = {};
 #pragma unroll
-                for (int x = 0; x < 8; ++x) acc[x] = 0.f;
+                for (int ks = 0; ks < 4; ++ks) {
+                    if (ks < 2 * (mb + 1)) {
+                        const float2 a01 = *reinterpret_cast<const float2*>(sTf + (32 + 16 * mb + g) * LDA + 32 + 8 * ks + 2 * t);
+                        const float2 a23 = *reinterpret_cast<const float2*>(sTf + (32 + 16 * mb + g + 8) * LDA + 32 + 8 * ks + 2 * t);
+                        const uint32_t af[4] = {tf32_rna(a01.x), tf32_rna(a23.x), tf32_rna(a01.y), tf32_rna(a23.y)};
 #pragma unroll
-                for (int i4 = 0; i4 < 2; ++i4) {
-                    const int ib = 8 * ih + 4 * i4;
-                    float yv[4];
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) yv[e] = sY[(16 * pr + ib + e) * LDY + c];
-#pragma unroll
-                    for (int x = 0; x < 8; ++x) {
-                        const float4 a4 = *reinterpret_cast<const float4*>(sTf + (hi + r0 + x) * LDA + hi + ib);
-                        acc[x] = fmaf(a4.x, yv[0], fmaf(a4.y, yv[1], fmaf(a4.z, yv[2], fmaf(a4.w, yv[3], acc[x]))));
-                    }
-                }
-#pragma unroll
-                for (int x = 0; x < 8; ++x) {
-                    acc[x] += __shfl_xor_sync(0xffffffffu, acc[x], 16);
-                    if (ih == 0) sTf[(hi + r0 + x) * LDA + lo + c] = -acc[x];
-                    else sTf[(lo + r0 + x) * LDA + hi + c] = 0.f;      // the upper-right 16-blocks are zero
-                }
-            }
-            named_bar_sync(1, 128);
-            {   // level 2: the 32-block (1,0)
-                const int r0 = 8 * warp, c = lane;
-                float acc[8];
-#pragma unroll
-                for (int x = 0; x < 8; ++x) acc[x] = 0.f;
-#pragma unroll 2
-                for (int i4 = 0; i4 < 8; ++i4) {
-                    float tv[4];
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) tv[e] = sTf[(4 * i4 + e) * LDA + c];
-#pragma unroll
-                    for (int x = 0; x < 8; ++x) {
-                        const float4 a4 = *reinterpret_cast<const float4*>(sA + (32 + r0 + x) * LDA + 4 * i4);
-                        acc[x] = fmaf(a4.x, tv[0], fmaf(a4.y, tv[1], fmaf(a4.z, tv[2], fmaf(a4.w, tv[3], acc[x]))));
-                    }
-                }
-#pragma unroll
-                for (int x = 0; x < 8; ++x) sY[(r0 + x) * LDY + c] = acc[x];
-                named_bar_sync(1, 128);
-#pragma unroll
-                for (int x = 0; x < 8; ++x) acc[x] = 0.f;
-                // T22 is lower triangular: row r of it ends at column r.  With the rows dealt out round robin
-                // (this warp owns rows warp, warp + 4, ...) row x of the warp needs the column blocks 0..x only,
-                // the same for every warp: 36 of the 64 (block, row) pairs.
-#pragma unroll
-                for (int i4 = 0; i4 < 8; ++i4) {
-                    float yv[4];
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) yv[e] = sY[(4 * i4 + e) * LDY + c];
-#pragma unroll
-                    for (int x = 0; x < 8; ++x) {
-                        if (x >= i4) {
-                            const float4 a4 = *reinterpret_cast<const float4*>(sTf + (32 + warp + 4 * x) * LDA + 32 + 4 * i4);
-                            acc[x] = fmaf(a4.x, yv[0], fmaf(a4.y, yv[1], fmaf(a4.z, yv[2], fmaf(a4.w, yv[3], acc[x]))));
+                        for (int q = 0; q < 4; ++q) {
+                            const uint32_t b0 = tf32_rna(sA[(32 + 8 * ks + 2 * t) * LDA + 8 * q + g]);
+                            const uint32_t b1 = tf32_rna(sA[(32 + 8 * ks + 2 * t + 1) * LDA + 8 * q + g]);
+                            mma_tf32(z[q], af, b0, b1);
                         }
                     }
                 }
+                float r[2][4] = {};
 #pragma unroll
-                for (int x = 0; x < 8; ++x) sTf[(32 + warp + 4 * x) * LDA + c] = -acc[x];
+                for (int ks = 0; ks < 4; ++ks) {
+                    if (ks >= 2 * nb) {
+                        const uint32_t af[4] = {tf32_rna(z[ks][0]), tf32_rna(z[ks][2]), tf32_rna(z[ks][1]), tf32_rna(z[ks][3])};
+#pragma unroll
+                        for (int q = 0; q < 2; ++q) {
+                            const uint32_t b0 = tf32_rna(sTf[(8 * ks + 2 * t) * LDA + 16 * nb + 8 * q + g]);
+                            const uint32_t b1 = tf32_rna(sTf[(8 * ks + 2 * t + 1) * LDA + 16 * nb + 8 * q + g]);
+                            mma_tf32(r[q], af, b0, b1);
+                        }
+                    }
+                }
+                named_bar_sync(1, 128);                    // every warp has read A21: overwrite it
+#pragma unroll
+                for (int q = 0; q < 2; ++q) {
+                    *reinterpret_cast<float2*>(sTf + (32 + 16 * mb + g) * LDA + 16 * nb + 8 * q + 2 * t) = make_float2(-r[q][0], -r[q][1]);
+                    *reinterpret_cast<float2*>(sTf + (32 + 16 * mb + g + 8) * LDA + 16 * nb + 8 * q + 2 * t) = make_float2(-r[q][2], -r[q][3]);
+                }
             }
             if (tp == 0) bulk_wait_read_all();                 // the P image has left the Q_lo tile
             named_bar_sync(1, 128);
@@ -655,19 +661,62 @@ struct ChainParams {
     int snap_every, nsnap;
 };
 
-template <bool DBG>
-__global__ void __launch_bounds__(CHAIN_THREADS, 1)
-gdn_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
-                 const __grid_constant__ CUtensorMap map_v, ChainParams p) {
-    extern __shared__ uint8_t smem_raw[];
-    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    uint8_t* sm = smem_raw + (base - smem_u32(smem_raw));
-    volatile uint32_t* sMisc = reinterpret_cast<volatile uint32_t*>(sm + CS_MISC);
-    Waiter w{base + CS_BARS, reinterpret_cast<volatile int*>(sm + CS_MISC + 4)};
+// One CTA's identity inside a kernel: aligned shared-memory base (address and pointer), tensor-memory base,
+// and the grid coordinates the stand-alone kernels take from blockIdx.
+struct Cta {
+    uint32_t base;
+    uint8_t* sm;
+    uint32_t tmem;
+    int dvb, h, z;
+};
+// Grid-level hand-over inside the merged scan kernel: `flag` is a counter in global memory that the CTAs of one
+// (sequence, head) raise when their part of a phase is written; a consumer waits (bounded) until it reads
+// `target`.  nullptr = no waiting (stand-alone kernels: the kernel boundary orders everything).
+struct Handover {
+    const int* flag;
+    int target;
+};
+__device__ __forceinline__ int ld_acquire_gpu(const int* p) {
+    int v;
+    asm volatile("ld.acquire.gpu.global.b32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+// One thread polls; returns false when the wait was given up (abort flag set, status raised).
+__device__ __forceinline__ bool handover_wait(const Handover& hv, volatile int* abort_flag) {
+    if (!hv.flag) return true;
+    const unsigned long long t0 = globaltimer_ns();
+    while (ld_acquire_gpu(hv.flag) < hv.target) {
+        if (*abort_flag) return false;
+        if (globaltimer_ns() - t0 > TIMEOUT_NS) {
+            *abort_flag = 1;
+            atomicCAS(&g_lean_status, 0, (int)GDN_ERR_TIMEOUT);
+            return false;
+        }
+        __nanosleep(40);
+    }
+    // data written with ordinary stores by other SMs is about to be read by bulk copies as well
+    asm volatile("fence.proxy.async;" ::: "memory");
+    return true;
+}
 
+__device__ __forceinline__ void chain_init_bars(const Waiter& w) {
+    for (uint32_t i = 0; i < 2; ++i) { mbar_init(w.bar(CB_FULLA0 + i), 1); mbar_init(w.bar(CB_FREEA0 + i), 2); }   // both issuers
+    mbar_init(w.bar(CB_U), 1); mbar_init(w.bar(CB_O1), 1);
+    for (uint32_t i = 0; i < 3; ++i) { mbar_init(w.bar(CB_FULLB0 + i), 1); mbar_init(w.bar(CB_FREEB0 + i), 1); }
+    mbar_init(w.bar(CB_V), 1); mbar_init(w.bar(CB_S), 1); mbar_init(w.bar(CB_O), 1);
+    mbar_init(w.bar(CB_SREADY), 128); mbar_init(w.bar(CB_VREADY), 128); mbar_init(w.bar(CB_OFREE), 128);
+}
+
+// Steps c and d for one CTA.  SCAN: called from the merged scan kernel (register budgets are set there, the
+// incoming state is awaited through `hv` and read past the L1 cache, since another SM wrote it in this launch).
+template <bool DBG, bool SCAN>
+__device__ __forceinline__ void chain_body(const CUtensorMap* map_q, const CUtensorMap* map_k, const CUtensorMap* map_v,
+                                           const ChainParams& p, const Cta& cta, const Waiter& w, const Handover& hv) {
+    const uint32_t base = cta.base, tmem = cta.tmem;
+    uint8_t* sm = cta.sm;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int dvb = blockIdx.x, h = blockIdx.y;
-    const int n = blockIdx.z / p.nseg, seg = blockIdx.z % p.nseg;
+    const int dvb = cta.dvb, h = cta.h;
+    const int n = cta.z / p.nseg, seg = cta.z % p.nseg;
     const int H = p.H, dv = p.dv;
     const SeqInfo sq = seq_info(p.cu, n, p.T);
     // this CTA walks chunks [seg * seg_chunks, ...) of the sequence
@@ -676,43 +725,31 @@ gdn_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     const int len = max(0, min(sq.len - cbeg * C, p.seg_chunks * C));
     const int nchunks = (len + C - 1) / C;
     const long slot0 = slot_base(sq.tok0, n) + cbeg;
-
-    if (tid == 0) {
-        for (uint32_t i = 0; i < 2; ++i) { mbar_init(w.bar(CB_FULLA0 + i), 1); mbar_init(w.bar(CB_FREEA0 + i), 2); }   // both issuers
-        mbar_init(w.bar(CB_U), 1); mbar_init(w.bar(CB_O1), 1);
-        for (uint32_t i = 0; i < 3; ++i) { mbar_init(w.bar(CB_FULLB0 + i), 1); mbar_init(w.bar(CB_FREEB0 + i), 1); }
-        mbar_init(w.bar(CB_V), 1); mbar_init(w.bar(CB_S), 1); mbar_init(w.bar(CB_O), 1);
-        mbar_init(w.bar(CB_SREADY), 128); mbar_init(w.bar(CB_VREADY), 128); mbar_init(w.bar(CB_OFREE), 128);
-        sMisc[1] = 0;
-        fence_mbar_init();
-    }
-    if (warp == 0) {
-        tmem_alloc(base + CS_MISC, CT_COLS);
-        tmem_relinquish();
-    }
-    tc_fence_before_sync();
-    __syncthreads();
-    tc_fence_after_sync();
-    const uint32_t tmem = sMisc[0];
-    pdl_wait();                         // scratch items and incoming states come from the kernels before this one
     const unsigned long long t_start = DBG ? globaltimer_ns() : 0ull;
     auto stamp = [&](int role, int c, int ev) {
-        if (DBG && p.dbg && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && c < 32)
+        if (DBG && p.dbg && dvb == 0 && h == 0 && cta.z == 0 && c < 32)
             p.dbg[(role * 32 + c) * 8 + ev] = (float)(globaltimer_ns() - t_start);
     };
     const size_t state_off = ((size_t)n * H + h) * DK * dv + (size_t)dvb * DVB;
-    const float* s_in = (seg == 0) ? (p.s0 ? p.s0 + state_off : nullptr)
-                                   : p.seg_sin + ((size_t)(n * p.nseg + seg) * H + h) * DK * dv + (size_t)dvb * DVB;
+    // With a split every segment, the first included, takes its incoming state from seg_sin (the combine
+    // kernel copied the caller's initial state there): nothing reads initial_state once this kernel runs,
+    // so final_state may alias it.
+    const float* s_in = p.seg_sin ? p.seg_sin + ((size_t)(n * p.nseg + seg) * H + h) * DK * dv + (size_t)dvb * DVB
+                                  : (p.s0 ? p.s0 + state_off : nullptr);
 
     if (warp < 4) {
         // =============================== chain warpgroup ===============================
-        setmaxnreg_inc<232>();
+        if (!SCAN) setmaxnreg_inc<232>();
         const int j = tid;
         const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
         float S[DK];
+        if (SCAN) {                                     // the combine phase of every slice of this head has been written
+            if (tid == 0) handover_wait(hv, w.abort_flag);
+            named_bar_sync(3, 128);
+        }
         if (s_in) {
 #pragma unroll
-            for (int m = 0; m < DK; ++m) S[m] = __ldg(s_in + (size_t)m * dv + j);
+            for (int m = 0; m < DK; ++m) S[m] = SCAN ? __ldcg(s_in + (size_t)m * dv + j) : __ldg(s_in + (size_t)m * dv + j);
         } else {
 #pragma unroll
             for (int m = 0; m < DK; ++m) S[m] = 0.f;
@@ -851,7 +888,7 @@ gdn_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         }
     } else {
         // =============================== control warpgroup ===============================
-        setmaxnreg_dec<56>();
+        if (!SCAN) setmaxnreg_dec<56>();
         if (warp == 8 && lane == 0) {
             // ---- MMA issuer of the sequential chain: v_new and the state update, nothing else ----
             // (issuing costs tens of nanoseconds per instruction; everything off the chain is
@@ -921,19 +958,19 @@ gdn_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             }
         } else if (warp == 9 && lane == 0) {
             // ---- TMA producer ----
-            prefetch_tensormap(&map_q);
-            prefetch_tensormap(&map_k);
-            prefetch_tensormap(&map_v);
+            prefetch_tensormap(map_q);
+            prefetch_tensormap(map_k);
+            prefetch_tensormap(map_v);
             for (int c = 0; c < nchunks; ++c) {
-                if (c == p.drop_chunk && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0) continue;
+                if (c == p.drop_chunk && dvb == 0 && h == 0 && cta.z == 0) continue;
                 const int tok = (int)(tok0 + (long)c * C);
                 const uint8_t* item = p.items + (size_t)((slot0 + c) * H + h) * ITEM_BYTES;
                 {   // ring B: V tile and (T diag(b))^T
                     const uint32_t sB = c % 3, bb = base + CS_B + sB * STAGE_B, full = w.bar(CB_FULLB0 + sB);
                     if (c >= 3) w.wait(CB_FREEB0 + sB, ((c / 3) - 1) & 1);
                     mbar_arrive_expect_tx(full, STAGE_B_TX);
-                    tma_load_3d(bb + ST_V, &map_v, dvb * DVB, h, tok, full);
-                    tma_load_3d(bb + ST_V + 8192, &map_v, dvb * DVB + 64, h, tok, full);
+                    tma_load_3d(bb + ST_V, map_v, dvb * DVB, h, tok, full);
+                    tma_load_3d(bb + ST_V + 8192, map_v, dvb * DVB + 64, h, tok, full);
                     bulk_load(bb + ST_T2, item + IT_T2, 8192, full);
                 }
                 {   // ring A: K/Q tiles, -W^T, P, and the gate vectors (own 4-deep ring, same barrier)
@@ -941,10 +978,10 @@ gdn_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                     if (c >= 2) w.wait(CB_FREEA0 + s, ((c >> 1) - 1) & 1);
                     mbar_arrive_expect_tx(full, STAGE_A_TX);
                     bulk_load(sb + ST_W, item + IT_W, 16384, full);
-                    tma_load_3d(sb + ST_KQ, &map_k, 0, h, tok, full);
-                    tma_load_3d(sb + ST_KQ + 8192, &map_q, 0, h, tok, full);
-                    tma_load_3d(sb + ST_KQ + 16384, &map_k, 64, h, tok, full);
-                    tma_load_3d(sb + ST_KQ + 24576, &map_q, 64, h, tok, full);
+                    tma_load_3d(sb + ST_KQ, map_k, 0, h, tok, full);
+                    tma_load_3d(sb + ST_KQ + 8192, map_q, 0, h, tok, full);
+                    tma_load_3d(sb + ST_KQ + 16384, map_k, 64, h, tok, full);
+                    tma_load_3d(sb + ST_KQ + 24576, map_q, 64, h, tok, full);
                     bulk_load(sb + ST_P, item + IT_P, 8192, full);
                     bulk_load(base + CS_GATES + (c & 3) * 1280, item + IT_GATES, 1280, full);
                 }
@@ -960,6 +997,34 @@ gdn_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             }
         }
     }
+}
+
+template <bool DBG>
+__global__ void __launch_bounds__(CHAIN_THREADS, 1)
+gdn_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
+                 const __grid_constant__ CUtensorMap map_v, ChainParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* sm = smem_raw + (base - smem_u32(smem_raw));
+    volatile uint32_t* sMisc = reinterpret_cast<volatile uint32_t*>(sm + CS_MISC);
+    Waiter w{base + CS_BARS, reinterpret_cast<volatile int*>(sm + CS_MISC + 4)};
+    const int warp = threadIdx.x >> 5;
+    if (threadIdx.x == 0) {
+        chain_init_bars(w);
+        sMisc[1] = 0;
+        fence_mbar_init();
+    }
+    if (warp == 0) {
+        tmem_alloc(base + CS_MISC, CT_COLS);
+        tmem_relinquish();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem = sMisc[0];
+    pdl_wait();                         // scratch items and incoming states come from the kernels before this one
+    const Cta cta{base, sm, tmem, (int)blockIdx.x, (int)blockIdx.y, (int)blockIdx.z};
+    chain_body<DBG, false>(&map_q, &map_k, &map_v, p, cta, w, Handover{nullptr, 0});
     tc_fence_before_sync();
     __syncthreads();
     if (warp == 0) {
@@ -983,6 +1048,7 @@ gdn_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
 // segment from its true incoming state.
 // =====================================================================================
 constexpr int SUM_THREADS = 384;
+constexpr uint32_t CMB_IMG = 65536;                         // M_seg^T per (segment, head): leading bf16 image | remainder image
 constexpr uint32_t SS_K = 0, SS_V = 16384, SS_W = 32768, SS_T2 = 49152, SS_GATES = 57344;
 constexpr uint32_t SUM_STAGE = 59392;                       // 58 KiB
 constexpr uint32_t SUM_STAGE_TX = 16384 + 16384 + 16384 + 8192 + 1280;
@@ -1003,24 +1069,32 @@ struct SummaryParams {
     const int32_t* cu;
     const uint8_t* items;
     float* seg_n;             // [B*nseg, H, d_k, d_v]   N_seg
-    float* seg_mt;            // [B*nseg, H, d_k(i), d_k(m)]  M_seg transposed
+    float* seg_mt;            // [B*nseg, H] x 64 KiB: M_seg^T as two bf16 operand images (leading part | remainder)
     int B, T, H, dv;
     int nseg, seg_chunks;
 };
 
-__global__ void __launch_bounds__(SUM_THREADS, 1)
-gdn_summary_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
-                   SummaryParams p) {
-    extern __shared__ uint8_t smem_raw[];
-    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    uint8_t* sm = smem_raw + (base - smem_u32(smem_raw));
-    volatile uint32_t* sMisc = reinterpret_cast<volatile uint32_t*>(sm + SUS_MISC);
-    Waiter w{base + SUS_BARS, reinterpret_cast<volatile int*>(sm + SUS_MISC + 4)};
+__device__ __forceinline__ void summary_init_bars(const Waiter& w, int ninst) {
+    for (uint32_t i = 0; i < SUM_STAGES; ++i) {
+        mbar_init(w.bar(SB_FULL0 + i), 1);
+        mbar_init(w.bar(SB_FREE0 + i), 129 * ninst);         // per instance: its issue thread and its warpgroup
+    }
+    for (uint32_t i = 0; i < 2; ++i) {
+        mbar_init(w.bar(SB_V0 + i), 1); mbar_init(w.bar(SB_S0 + i), 1);
+        mbar_init(w.bar(SB_SREADY0 + i), 128); mbar_init(w.bar(SB_VREADY0 + i), 128);
+    }
+}
 
+// Segment summary (M_seg, N_seg) of one CTA; cta.z = sequence * (nseg - 1) + segment.
+template <bool SCAN>
+__device__ __forceinline__ void summary_body(const CUtensorMap* map_k, const CUtensorMap* map_v, const SummaryParams& p,
+                                             const Cta& cta, const Waiter& w) {
+    const uint32_t base = cta.base, tmem = cta.tmem;
+    uint8_t* sm = cta.sm;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int dvb = blockIdx.x, h = blockIdx.y;
+    const int dvb = cta.dvb, h = cta.h;
     const int nsum = p.nseg - 1;                      // the last segment needs no summary
-    const int n = blockIdx.z / nsum, seg = blockIdx.z % nsum;
+    const int n = cta.z / nsum, seg = cta.z % nsum;
     const int H = p.H, dv = p.dv;
     const SeqInfo sq = seq_info(p.cu, n, p.T);
     const int cbeg = seg * p.seg_chunks;
@@ -1031,32 +1105,9 @@ gdn_summary_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
     const bool with_m = (dvb == 0);                   // M_seg does not depend on the value columns
     const int ninst = with_m ? 2 : 1;
 
-    if (tid == 0) {
-        for (uint32_t i = 0; i < SUM_STAGES; ++i) {
-            mbar_init(w.bar(SB_FULL0 + i), 1);
-            mbar_init(w.bar(SB_FREE0 + i), 129 * ninst);         // per instance: its issue thread and its warpgroup
-        }
-        for (uint32_t i = 0; i < 2; ++i) {
-            mbar_init(w.bar(SB_V0 + i), 1); mbar_init(w.bar(SB_S0 + i), 1);
-            mbar_init(w.bar(SB_SREADY0 + i), 128); mbar_init(w.bar(SB_VREADY0 + i), 128);
-        }
-        sMisc[1] = 0;
-        fence_mbar_init();
-    }
-    if (warp == 0) {
-        tmem_alloc(base + SUS_MISC, SUM_COLS);
-        tmem_relinquish();
-    }
-    tc_fence_before_sync();
-    __syncthreads();
-    tc_fence_after_sync();
-    const uint32_t tmem = sMisc[0];
-    pdl_trigger();
-    pdl_wait();                         // the scratch items come from the prepare kernel
-
     if (warp < 8) {
         // ======================= two chain warpgroups: values (0) and identity (1) =======================
-        setmaxnreg_inc<224>();
+        if (!SCAN) setmaxnreg_inc<224>();
         const int inst = warp >> 2;
         const int j = tid & 127;
         const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
@@ -1123,14 +1174,31 @@ gdn_summary_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
 #pragma unroll
                 for (int m = 0; m < DK; ++m) dst[(size_t)m * dv] = S[m];
             } else {
-                float4* dst = reinterpret_cast<float4*>(p.seg_mt + sidx * DK * DK + (size_t)j * DK);  // [i = j][m]
+                // M_seg^T leaves as two bf16 operand images (leading part, remainder): row i = j holds
+                // M_seg[m][i] for all m, in the layout the combine kernel's MMAs read (128-byte swizzle,
+                // blocks of 64 rows x 64 columns).  Leading part + remainder carry 16 mantissa bits.
+                uint8_t* img = reinterpret_cast<uint8_t*>(p.seg_mt) + sidx * CMB_IMG + (uint32_t)(j >> 6) * 16384;
+                const uint32_t r = (uint32_t)j & 63u;
 #pragma unroll
-                for (int m4 = 0; m4 < DK / 4; ++m4) dst[m4] = make_float4(S[4 * m4], S[4 * m4 + 1], S[4 * m4 + 2], S[4 * m4 + 3]);
+                for (int mh = 0; mh < 2; ++mh)
+#pragma unroll
+                    for (int ch = 0; ch < 8; ++ch) {
+                        uint32_t hi[4], lo[4];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const float x0 = S[64 * mh + 8 * ch + 2 * e], x1 = S[64 * mh + 8 * ch + 2 * e + 1];
+                            hi[e] = pack_bf16(x0, x1);
+                            lo[e] = pack_bf16(x0 - __uint_as_float(hi[e] << 16), x1 - __uint_as_float(hi[e] & 0xffff0000u));
+                        }
+                        uint8_t* dst = img + mh * 8192 + swz(r, ch);
+                        st_global_v4(dst, hi[0], hi[1], hi[2], hi[3]);
+                        st_global_v4(dst + CMB_IMG / 2, lo[0], lo[1], lo[2], lo[3]);
+                    }
             }
         }
     } else {
         // =============================== control warpgroup ===============================
-        setmaxnreg_dec<56>();
+        if (!SCAN) setmaxnreg_dec<56>();
         if ((warp == 8 || warp == 10) && lane == 0) {
             // ---- one MMA issue thread per chain instance (they are independent) ----
             const int inst = (warp == 8) ? 0 : 1;
@@ -1165,8 +1233,8 @@ gdn_summary_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
                 }
             }
         } else if (warp == 9 && lane == 0) {
-            prefetch_tensormap(&map_k);
-            prefetch_tensormap(&map_v);
+            prefetch_tensormap(map_k);
+            prefetch_tensormap(map_v);
             for (int c = 0; c < nchunks; ++c) {
                 const uint32_t s = c % SUM_STAGES, sb = base + s * SUM_STAGE;
                 if (c >= (int)SUM_STAGES) w.wait(SB_FREE0 + s, ((c / SUM_STAGES) - 1) & 1);
@@ -1174,10 +1242,10 @@ gdn_summary_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
                 const int tok = (int)(tok0 + (long)c * C);
                 const uint8_t* item = p.items + (size_t)((slot0 + c) * H + h) * ITEM_BYTES;
                 mbar_arrive_expect_tx(full, SUM_STAGE_TX);
-                tma_load_3d(sb + SS_K, &map_k, 0, h, tok, full);
-                tma_load_3d(sb + SS_K + 8192, &map_k, 64, h, tok, full);
-                tma_load_3d(sb + SS_V, &map_v, dvb * DVB, h, tok, full);
-                tma_load_3d(sb + SS_V + 8192, &map_v, dvb * DVB + 64, h, tok, full);
+                tma_load_3d(sb + SS_K, map_k, 0, h, tok, full);
+                tma_load_3d(sb + SS_K + 8192, map_k, 64, h, tok, full);
+                tma_load_3d(sb + SS_V, map_v, dvb * DVB, h, tok, full);
+                tma_load_3d(sb + SS_V + 8192, map_v, dvb * DVB + 64, h, tok, full);
                 bulk_load(sb + SS_W, item + IT_W, 16384, full);
                 bulk_load(sb + SS_T2, item + IT_T2, 8192, full);
                 bulk_load(sb + SS_GATES, item + IT_GATES, 1280, full);
@@ -1191,6 +1259,34 @@ gdn_summary_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
             }
         }
     }
+}
+
+__global__ void __launch_bounds__(SUM_THREADS, 1)
+gdn_summary_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
+                   SummaryParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* sm = smem_raw + (base - smem_u32(smem_raw));
+    volatile uint32_t* sMisc = reinterpret_cast<volatile uint32_t*>(sm + SUS_MISC);
+    Waiter w{base + SUS_BARS, reinterpret_cast<volatile int*>(sm + SUS_MISC + 4)};
+    const int warp = threadIdx.x >> 5;
+    if (threadIdx.x == 0) {
+        summary_init_bars(w, blockIdx.x == 0 ? 2 : 1);
+        sMisc[1] = 0;
+        fence_mbar_init();
+    }
+    if (warp == 0) {
+        tmem_alloc(base + SUS_MISC, SUM_COLS);
+        tmem_relinquish();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem = sMisc[0];
+    pdl_trigger();
+    pdl_wait();                         // the scratch items come from the prepare kernel
+    const Cta cta{base, sm, tmem, (int)blockIdx.x, (int)blockIdx.y, (int)blockIdx.z};
+    summary_body<false>(&map_k, &map_v, p, cta, w);
     tc_fence_before_sync();
     __syncthreads();
     if (warp == 0) {
@@ -1199,105 +1295,322 @@ gdn_summary_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
     }
 }
 
-// S_in[p+1] = M_p S_in[p] + N_p in fp32, p = 0 .. nseg-2; one CTA per (sequence, head, 16 value
-// columns).  M_p^T (64 KiB) is brought into shared memory by bulk copies, two segments ahead,
-// so the only serial cost per segment is the 128 x 128 x 16 product itself.
-constexpr int CMB_COLS = 16;
-constexpr int CMB_THREADS = 512;                       // 4 groups along the contraction x (32 x 4) tiles of 4 x 4
-constexpr uint32_t CMB_MT_BYTES = DK * DK * 4;
-constexpr uint32_t CMB_BUFS = 2;
-constexpr uint32_t CMB_S_BYTES = DK * CMB_COLS * 4;
-constexpr int CMB_LDP = CMB_COLS + 4;                  // padded row of the partial sums (bank spread)
-constexpr uint32_t CMB_SMEM = CMB_BUFS * CMB_MT_BYTES + CMB_S_BYTES + 4 * DK * CMB_LDP * 4 + 64 + 128;
+// S_in[p+1] = M_p S_in[p] + N_p, p = 0 .. nseg-2; one CTA per (sequence, head, CMB_COLS value columns).
+// Each hop is a 128 x CMB_COLS x 128 product on the tensor core with both factors split into a leading bf16
+// part and a bf16 remainder (hi*hi + lo*hi + hi*lo, fp32 accumulation: 16 mantissa bits per factor), so
+// the hops cost MMA round trips instead of fp32 FMAs.  A = M_p as the two operand images the summary kernel
+// wrote (bulk copies, three segments ahead); B = the state slice, written to shared memory by the
+// thread that owns each row; D in tensor memory.  The incoming state of segment 0 is copied to seg_sin as
+// well, so that no later kernel reads the caller's initial_state (which final_state may alias).
+constexpr int CMB_COLS = 16;                           // value columns per CTA.  Measured on the 10240-token workload: a hop takes
+                                                       // about 1.0 us + 0.05 us per column (each thread converts, stores and
+                                                       // reloads its own row), so narrow slices on many SMs win
+constexpr int CMB_THREADS = 160;                       // warps 0-3: one state row per thread; warp 4: copies and MMA issue
+constexpr uint32_t CMB_STAGES = 3;
+constexpr uint32_t CMB_BIMG = CMB_COLS * 256;          // one image of the state slice: [column][row m], two 64-row blocks
+constexpr uint32_t CM_B = CMB_STAGES * CMB_IMG;        // state slice images: leading part | remainder
+constexpr uint32_t CM_BARS = CM_B + 2 * CMB_BIMG;
+constexpr uint32_t CM_MISC = CM_BARS + 16 * 8;
+constexpr uint32_t CMB_SMEM = CM_MISC + 64 + 1024;
+constexpr uint32_t CMB_TCOLS = CMB_COLS < 32 ? 32 : CMB_COLS;
+enum MBar : uint32_t { MB_FULL0 = 0, MB_FREE0 = 3, MB_BREADY = 6, MB_D = 7 };
+constexpr uint32_t ID_CMB = make_idesc(128, CMB_COLS, kFmtBF16, kFmtBF16, kMajorMN, kMajorK);
+
 struct CombineParams {
     const float* s0;          // [B, H, d_k, d_v] or nullptr
     const float* seg_n;
-    const float* seg_mt;
+    const float* seg_mt;      // per (sequence, segment, head): leading | remainder image of M_seg^T
     float* seg_sin;
     int H, dv, nseg;
 };
 
-__global__ void __launch_bounds__(CMB_THREADS) gdn_combine_kernel(CombineParams p) {
-    extern __shared__ uint8_t smem_raw[];
-    const uint32_t base = (smem_u32(smem_raw) + 127u) & ~127u;
-    uint8_t* sm = smem_raw + (base - smem_u32(smem_raw));
-    const float* sMt = reinterpret_cast<const float*>(sm);                                   // [CMB_BUFS][i][m]
-    float (*sS)[CMB_COLS] = reinterpret_cast<float (*)[CMB_COLS]>(sm + CMB_BUFS * CMB_MT_BYTES);
-    float* sPart = reinterpret_cast<float*>(sm + CMB_BUFS * CMB_MT_BYTES + CMB_S_BYTES);     // [4][m][16]
-    const uint32_t misc = CMB_BUFS * CMB_MT_BYTES + CMB_S_BYTES + 4 * DK * CMB_LDP * 4;
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(sm + misc + 32);
-    Waiter w{base + misc, abort_flag};
+__device__ __forceinline__ void combine_init_bars(const Waiter& w) {
+    for (uint32_t i = 0; i < CMB_STAGES; ++i) { mbar_init(w.bar(MB_FULL0 + i), 1); mbar_init(w.bar(MB_FREE0 + i), 1); }
+    mbar_init(w.bar(MB_BREADY), 128);
+    mbar_init(w.bar(MB_D), 1);
+}
 
-    const int tid = threadIdx.x;
-    const int j0 = blockIdx.x * CMB_COLS, h = blockIdx.y, n = blockIdx.z;
-    const int H = p.H, dv = p.dv;
-    // product phase: a warp covers 8 row tiles x 4 column tiles, so its M loads touch one 128-byte line
-    const int kg = tid >> 7, ct = tid & 3, mt4 = ((tid >> 2) & 7) + 8 * ((tid >> 5) & 3);
-    const int rm = tid >> 2, rc = (tid & 3) * 4;                       // reduction phase: 4 outputs of row rm
-    auto load_mt = [&](int seg) {
-        const uint32_t buf = seg % CMB_BUFS, full = w.bar(buf);
-        const uint8_t* src = reinterpret_cast<const uint8_t*>(p.seg_mt + ((size_t)(n * p.nseg + seg) * H + h) * DK * DK);
-        mbar_arrive_expect_tx(full, CMB_MT_BYTES);
+// The hops of one column slice (cta.dvb = slice, cta.z = sequence).  Warps 0-3 own the rows, lane 0 of warp
+// `issue_warp` copies and issues.  SCAN: inside the merged scan kernel the summaries were written by other SMs
+// during this launch, so they are read past the L1 cache and no programmatic-launch wait applies.
+template <bool SCAN>
+__device__ __forceinline__ void combine_body(const CombineParams& p, const Cta& cta, const Waiter& w, int issue_warp) {
+    const uint32_t base = cta.base, tmem = cta.tmem;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int j0 = cta.dvb * CMB_COLS, h = cta.h, n = cta.z;
+    const int H = p.H, dv = p.dv, nhops = p.nseg - 1;
+    auto seg_off = [&](int seg) { return ((size_t)(n * p.nseg + seg) * H + h) * DK * dv; };
+
+    if (warp < 4) {
+        // ---- thread m owns row m of the slice ----
+        const int m = tid;
+        const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
+        float s[CMB_COLS];
+        if (p.s0) {   // the initial state is an input of the call: it may be read before the predecessor has finished
+            const float4* src = reinterpret_cast<const float4*>(p.s0 + (((size_t)n * H + h) * DK + m) * dv + j0);
 #pragma unroll
-        for (uint32_t q = 0; q < 4; ++q)
-            bulk_load(base + buf * CMB_MT_BYTES + q * 16384, src + q * 16384, 16384, full);
-    };
-    if (tid == 0) {
-        for (uint32_t i = 0; i < CMB_BUFS; ++i) mbar_init(w.bar(i), 1);
-        *abort_flag = 0;
+            for (int q = 0; q < CMB_COLS / 4; ++q) { const float4 x = __ldg(src + q); s[4 * q] = x.x; s[4 * q + 1] = x.y; s[4 * q + 2] = x.z; s[4 * q + 3] = x.w; }
+        } else {
+#pragma unroll
+            for (int j = 0; j < CMB_COLS; ++j) s[j] = 0.f;
+        }
+        if (!SCAN) pdl_wait();          // M_seg, N_seg come from the summary kernel
+        auto store_sin = [&](int seg) {
+            float4* dst = reinterpret_cast<float4*>(p.seg_sin + seg_off(seg) + (size_t)m * dv + j0);
+#pragma unroll
+            for (int q = 0; q < CMB_COLS / 4; ++q) dst[q] = make_float4(s[4 * q], s[4 * q + 1], s[4 * q + 2], s[4 * q + 3]);
+        };
+        // element (column j, row m) of the K-major B images: the two 64-row blocks of m are CMB_COLS * 128 bytes apart
+        const uint32_t bcol = base + CM_B + (uint32_t)(m >> 6) * (CMB_COLS * 128) + (uint32_t)(m & 7) * 2;
+        const uint32_t bchunk = (uint32_t)(m & 63) >> 3;
+        for (int seg = 0; seg < nhops; ++seg) {
+            float4 nv[CMB_COLS / 4];
+            const float4* nsrc = reinterpret_cast<const float4*>(p.seg_n + seg_off(seg) + (size_t)m * dv + j0);
+#pragma unroll
+            for (int q = 0; q < CMB_COLS / 4; ++q) nv[q] = SCAN ? __ldcg(nsrc + q) : __ldg(nsrc + q);
+#pragma unroll
+            for (int j = 0; j < CMB_COLS; ++j) {
+                const __nv_bfloat16 hi = __float2bfloat16_rn(s[j]);
+                const __nv_bfloat16 lo = __float2bfloat16_rn(s[j] - __bfloat162float(hi));
+                const uint32_t addr = bcol + (uint32_t)j * 128 + ((bchunk ^ ((uint32_t)j & 7u)) << 4);
+                asm volatile("st.shared.b16 [%0], %1;" ::"r"(addr), "h"(*reinterpret_cast<const unsigned short*>(&hi)) : "memory");
+                asm volatile("st.shared.b16 [%0], %1;" ::"r"(addr + CMB_BIMG), "h"(*reinterpret_cast<const unsigned short*>(&lo)) : "memory");
+            }
+            fence_proxy_async_smem();
+            tc_fence_before_sync();
+            mbar_arrive(w.bar(MB_BREADY));
+            store_sin(seg);              // S_in of this segment drains while the product runs
+            w.wait_hot(MB_D, seg & 1);
+            tc_fence_after_sync();
+#pragma unroll
+            for (int q = 0; q < CMB_COLS / 16; ++q) {
+                uint32_t d[16];
+                tmem_ld16(tmem + lane_base + 16 * q, d);
+                tmem_wait_ld();
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const float4 x = nv[4 * q + e];
+                    s[16 * q + 4 * e + 0] = __uint_as_float(d[4 * e + 0]) + x.x;
+                    s[16 * q + 4 * e + 1] = __uint_as_float(d[4 * e + 1]) + x.y;
+                    s[16 * q + 4 * e + 2] = __uint_as_float(d[4 * e + 2]) + x.z;
+                    s[16 * q + 4 * e + 3] = __uint_as_float(d[4 * e + 3]) + x.w;
+                }
+            }
+        }
+        store_sin(nhops);
+    } else if (warp == issue_warp && lane == 0) {
+        // ---- bulk copies of the M images and MMA issue ----
+        if (!SCAN) pdl_wait();
+        auto load_m = [&](int seg) {
+            const uint32_t st = seg % CMB_STAGES, full = w.bar(MB_FULL0 + st);
+            const uint8_t* src = reinterpret_cast<const uint8_t*>(p.seg_mt) + ((size_t)(n * p.nseg + seg) * H + h) * CMB_IMG;
+            mbar_arrive_expect_tx(full, CMB_IMG);
+#pragma unroll
+            for (uint32_t q = 0; q < 4; ++q) bulk_load(base + st * CMB_IMG + q * 16384, src + q * 16384, 16384, full);
+        };
+        for (int sg = 0; sg < (int)CMB_STAGES && sg < nhops; ++sg) load_m(sg);
+        const uint64_t dB0 = make_smem_desc(base + CM_B, 16, 1024);
+        for (int seg = 0; seg < nhops; ++seg) {
+            const uint32_t st = seg % CMB_STAGES, ma = base + st * CMB_IMG;
+            w.wait_hot(MB_FULL0 + st, (seg / CMB_STAGES) & 1);
+            w.wait_hot(MB_BREADY, seg & 1);
+            tc_fence_after_sync();
+#pragma unroll
+            for (uint32_t prod = 0; prod < 3; ++prod) {          // hi*hi, lo*hi, hi*lo
+                const uint32_t aoff = (prod == 1) ? CMB_IMG / 2 : 0u, boff = (prod == 2) ? CMB_BIMG : 0u;
+#pragma unroll
+                for (uint32_t ks = 0; ks < 8; ++ks)
+                    mma_ss(tmem, make_smem_desc(ma + aoff + (ks >> 2) * 16384 + (ks & 3) * 2048, 8192, 1024),
+                           dB0 + (uint64_t)((boff + (ks >> 2) * (CMB_COLS * 128) + (ks & 3) * 32) >> 4), ID_CMB, (prod | ks) ? 1u : 0u);
+            }
+            mma_commit(w.bar(MB_D));
+            mma_commit(w.bar(MB_FREE0 + st));
+            if (seg + (int)CMB_STAGES < nhops) {
+                w.wait(MB_FREE0 + st, (seg / CMB_STAGES) & 1);   // the tensor core has read this stage
+                load_m(seg + CMB_STAGES);
+            }
+        }
+        if (*w.abort_flag) {             // let copies in flight land before shared memory is released (bounded)
+            const unsigned long long t0 = globaltimer_ns();
+            for (int seg = max(0, nhops - (int)CMB_STAGES); seg < nhops; ++seg)
+                while (!mbar_try_wait(w.bar(MB_FULL0 + seg % CMB_STAGES), (seg / CMB_STAGES) & 1) &&
+                       globaltimer_ns() - t0 < TIMEOUT_NS) {}
+        }
+    }
+}
+
+__global__ void __launch_bounds__(CMB_THREADS, 1) gdn_combine_kernel(CombineParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* sm = smem_raw + (base - smem_u32(smem_raw));
+    volatile uint32_t* sMisc = reinterpret_cast<volatile uint32_t*>(sm + CM_MISC);
+    Waiter w{base + CM_BARS, reinterpret_cast<volatile int*>(sm + CM_MISC + 4)};
+    const int warp = threadIdx.x >> 5;
+    if (threadIdx.x == 0) {
+        combine_init_bars(w);
+        sMisc[1] = 0;
         fence_mbar_init();
     }
-    for (int idx = tid; idx < DK * CMB_COLS; idx += CMB_THREADS) {
-        const int i = idx / CMB_COLS, j = idx % CMB_COLS;
-        sS[i][j] = p.s0 ? p.s0[(((size_t)n * H + h) * DK + i) * dv + j0 + j] : 0.f;
+    if (warp == 0) {
+        tmem_alloc(base + CM_MISC, CMB_TCOLS);
+        tmem_relinquish();
     }
-    pdl_trigger();
-    pdl_wait();                         // M_seg, N_seg come from the summary kernel (the initial state loaded above is an input)
+    tc_fence_before_sync();
     __syncthreads();
-    if (tid == 0)
-        for (int sg = 0; sg < (int)CMB_BUFS && sg + 1 < p.nseg; ++sg) load_mt(sg);
-    auto n_ptr = [&](int seg) {
-        return p.seg_n + (((size_t)(n * p.nseg + seg) * H + h) * DK + rm) * dv + j0 + rc;
+    tc_fence_after_sync();
+    const uint32_t tmem = sMisc[0];
+    pdl_trigger();
+    const Cta cta{base, sm, tmem, (int)blockIdx.x, (int)blockIdx.y, (int)blockIdx.z};
+    combine_body<false>(p, cta, w, 4);
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 0) {
+        tc_fence_after_sync();
+        tmem_dealloc(tmem, CMB_TCOLS);
+    }
+}
+
+// =====================================================================================
+// merged scan kernel: summary, combination and chain of a split sequence in ONE launch
+//
+// The three phases of the sequence split are latency chains of a few dozen microseconds each, and every
+// kernel boundary between them costs a launch, a set-up (barriers, tensor memory, first loads) and a drain.
+// Here one CTA per (sequence, head, segment) stays resident and runs all three phases; the hand-over between
+// phases goes through two counters per (sequence, head) in global memory:
+//   phase 1  segment summary (M_seg, N_seg) of its own segment           -> raises counter 0
+//   phase 2  waits for counter 0 = nseg - 1, then runs the hops of one 16-column slice of the state
+//            (CTAs seg, seg + nseg, ... take the slices)                   -> raises counter 1
+//   phase 3  its operand ring is filled at once; the chain warpgroup waits for counter 1 = number of slice
+//            owners, loads the incoming state of its segment and walks its chunks
+// Every wait on a counter is bounded like the mbarrier waits (status GDN_ERR_TIMEOUT, abort flag, all roles
+// fall through).  The grid must be co-resident (one CTA per SM): the host launches this kernel only when
+// sequences x heads x segments <= #SMs, otherwise the three stand-alone kernels run.  The counters are zero
+// before the launch and zero again after it (the last CTA of a head to get past both waits clears them), so a
+// captured launch can be replayed.
+// =====================================================================================
+constexpr int SCAN_THREADS = 384;
+constexpr uint32_t SC_BARS1 = CS_BARS;                 // behind the largest data layout (the chain phase's)
+constexpr uint32_t SC_BARS2 = SC_BARS1 + 24 * 8;
+constexpr uint32_t SC_BARS3 = SC_BARS2 + 16 * 8;
+constexpr uint32_t SC_MISC = SC_BARS3 + 24 * 8;
+constexpr uint32_t SCAN_SMEM = SC_MISC + 64 + 1024;
+static_assert(SUS_BARS <= CS_BARS && CM_BARS <= CS_BARS, "phase layouts must end before the barrier area");
+static_assert(SCAN_SMEM <= 232448, "shared memory per CTA");
+constexpr int SCAN_FLAG_INTS = 4;                      // per (sequence, head): summaries, slices, CTAs done, pad
+
+struct ScanParams {
+    SummaryParams sp;
+    CombineParams cb;
+    ChainParams cp;
+    int* flags;               // [B * H][4], zero before and after every launch
+};
+
+__device__ __forceinline__ void mbar_inval(uint32_t bar) {
+    asm volatile("mbarrier.inval.shared::cta.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+template <bool DBG>
+__global__ void __launch_bounds__(SCAN_THREADS, 1)
+gdn_scan_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
+                const __grid_constant__ CUtensorMap map_v, ScanParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* sm = smem_raw + (base - smem_u32(smem_raw));
+    volatile uint32_t* sMisc = reinterpret_cast<volatile uint32_t*>(sm + SC_MISC);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(sm + SC_MISC + 4);
+    const Waiter w1{base + SC_BARS1, abort_flag}, w2{base + SC_BARS2, abort_flag}, w3{base + SC_BARS3, abort_flag};
+
+    const int tid = threadIdx.x, warp = tid >> 5;
+    const int nseg = p.cp.nseg, H = p.cp.H;
+    const int h = blockIdx.y, n = blockIdx.z / nseg, seg = blockIdx.z % nseg;
+    int* fl = p.flags + (size_t)(n * H + h) * SCAN_FLAG_INTS;
+    const int nslices = p.cp.dv / CMB_COLS;
+    const int nowners = nseg < nslices ? nseg : nslices;
+
+    if (tid == 0) {
+        summary_init_bars(w1, 2);
+        combine_init_bars(w2);
+        chain_init_bars(w3);
+        sMisc[1] = 0;
+        fence_mbar_init();
+    }
+    if (warp == 0) {
+        tmem_alloc(base + SC_MISC, 512);
+        tmem_relinquish();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem = sMisc[0];
+    pdl_wait();                         // the scratch items come from the prepare kernel
+    auto stamp = [&](int ev) {
+        if (DBG && p.cp.dbg && tid == 0 && h == 0 && n == 0 && seg < 16)
+            p.cp.dbg[512 + seg * 16 + ev] = (float)(globaltimer_ns() & 0xFFFFFFull);
     };
-    float4 nv = make_float4(0.f, 0.f, 0.f, 0.f);
-    if (p.nseg > 1) nv = __ldg(reinterpret_cast<const float4*>(n_ptr(0)));
-    for (int seg = 0; seg + 1 < p.nseg; ++seg) {
-        const float4 ncur = nv;
-        if (seg + 2 < p.nseg) nv = __ldg(reinterpret_cast<const float4*>(n_ptr(seg + 1)));   // one hop ahead
-        w.wait(seg % CMB_BUFS, (seg / CMB_BUFS) & 1);
-        const float* mt = sMt + (seg % CMB_BUFS) * DK * DK + 4 * mt4;
-        float acc[4][4];
-#pragma unroll
-        for (int r = 0; r < 4; ++r)
-#pragma unroll
-            for (int c = 0; c < 4; ++c) acc[r][c] = 0.f;
-#pragma unroll 8
-        for (int ii = 0; ii < 32; ++ii) {
-            const int i = kg * 32 + ii;
-            const float4 a4 = *reinterpret_cast<const float4*>(mt + i * DK);
-            const float4 s4 = *reinterpret_cast<const float4*>(&sS[i][4 * ct]);
-            const float av[4] = {a4.x, a4.y, a4.z, a4.w}, sv[4] = {s4.x, s4.y, s4.z, s4.w};
-#pragma unroll
-            for (int r = 0; r < 4; ++r)
-#pragma unroll
-                for (int c = 0; c < 4; ++c) acc[r][c] = fmaf(av[r], sv[c], acc[r][c]);
+    // The three phases, run by every warp.  The code is instantiated once per warpgroup role below, each copy
+    // behind that role's register budget, so the phase bodies (which branch on the warp index themselves)
+    // reduce to the one role; CTA-wide synchronisation therefore uses a named barrier, not __syncthreads.
+    auto cta_sync = [&]() { named_bar_sync(4, SCAN_THREADS); };
+    auto phases = [&]() {
+        stamp(0);
+        // ---------------- phase 1: summary of this segment (the last segment needs none) ----------------
+        if (seg < nseg - 1) {
+            const Cta c1{base, sm, tmem, 0, h, n * (nseg - 1) + seg};
+            summary_body<true>(&map_k, &map_v, p.sp, c1, w1);
+            __threadfence();
+            tc_fence_before_sync();
+            cta_sync();
+            tc_fence_after_sync();
+            if (tid == 0) { __threadfence(); atomicAdd(fl + 0, 1); }
         }
-#pragma unroll
-        for (int r = 0; r < 4; ++r)
-            *reinterpret_cast<float4*>(sPart + (kg * DK + 4 * mt4 + r) * CMB_LDP + 4 * ct) =
-                make_float4(acc[r][0], acc[r][1], acc[r][2], acc[r][3]);
-        __syncthreads();                               // partial products done; sS and this M buffer are free
-        if (tid == 0 && seg + (int)CMB_BUFS < p.nseg - 1) load_mt(seg + CMB_BUFS);
-        float4 o = ncur;
-#pragma unroll
-        for (int g = 0; g < 4; ++g) {
-            const float4 q = *reinterpret_cast<const float4*>(sPart + (g * DK + rm) * CMB_LDP + rc);
-            o.x += q.x; o.y += q.y; o.z += q.z; o.w += q.w;
+        stamp(1);
+        // ---------------- phase 2: the hops of this CTA's column slices ----------------
+        if (seg < nslices) {
+            if (tid == 0) handover_wait(Handover{fl + 0, nseg - 1}, abort_flag);
+            cta_sync();
+            stamp(2);
+            for (int slice = seg; slice < nslices; slice += nseg) {
+                if (slice != seg) {     // barriers of the previous slice have advanced: start them afresh
+                    cta_sync();
+                    if (tid == 0) {
+                        for (uint32_t i = 0; i < 8; ++i) mbar_inval(w2.bar(i));
+                        combine_init_bars(w2);
+                        fence_mbar_init();
+                    }
+                    cta_sync();
+                }
+                const Cta c2{base, sm, tmem, slice, h, n};
+                combine_body<true>(p.cb, c2, w2, 8);
+                tc_fence_before_sync();
+            }
+            __threadfence();
+            cta_sync();
+            tc_fence_after_sync();
+            if (tid == 0) { __threadfence(); atomicAdd(fl + 1, 1); }
         }
-        *reinterpret_cast<float4*>(&sS[rm][rc]) = o;
-        __syncthreads();
-        // the global store drains while the next segment is being computed
-        *reinterpret_cast<float4*>(p.seg_sin + (((size_t)(n * p.nseg + seg + 1) * H + h) * DK + rm) * dv + j0 + rc) = o;
+        stamp(3);
+        // ---------------- phase 3: chain over this segment's chunks ----------------
+        const Cta c3{base, sm, tmem, 0, h, (int)blockIdx.z};
+        chain_body<DBG, true>(&map_q, &map_k, &map_v, p.cp, c3, w3, Handover{fl + 1, nowners});
+        stamp(4);
+        tc_fence_before_sync();
+        cta_sync();
+    };
+    // register budgets: warpgroup 0 holds a 128-value fp32 row per thread in all three phases (232), warpgroup 1
+    // the identity chain of the summary and the epilogue of the chain phase (216), warpgroup 2 issues and copies (56)
+    if (warp < 4) { setmaxnreg_inc<232>(); phases(); }
+    else if (warp < 8) { setmaxnreg_inc<216>(); phases(); }
+    else { setmaxnreg_dec<56>(); phases(); }
+    if (tid == 0) {                     // the last CTA of this head to get here clears the counters
+        __threadfence();
+        if (atomicAdd(fl + 2, 1) == nseg - 1) {
+            fl[0] = 0; fl[1] = 0; fl[2] = 0;
+            __threadfence();
+        }
+    }
+    if (warp == 0) {
+        tc_fence_after_sync();
+        tmem_dealloc(tmem, 512);
     }
 }
 
@@ -1325,7 +1638,11 @@ static void plan_split(int B, int T, int H, int d_v, bool packed, int num_sms, i
 }
 constexpr int kMaxSeg = 16;
 
-constexpr size_t kWorkspaceHeader = 256;     // the prepare kernel's item ticket lives in front of the items
+// In front of the items: the prepare kernel's item ticket (two ints) and, from int 16 on, the scan kernel's
+// counters (four ints per (sequence, head)).  All of it reads zero before a call and zero again after it.
+constexpr size_t kWorkspaceHeader = 4096;
+constexpr int kScanFlagOffset = 16;
+constexpr long kMaxScanChains = (long)(kWorkspaceHeader / sizeof(int) - kScanFlagOffset) / SCAN_FLAG_INTS;
 
 // The ticket must read zero before the first launch; every launch leaves it zero again.
 int lean_init_workspace(void* workspace) {
@@ -1348,19 +1665,54 @@ static void launch_after(void (*kernel)(KArgs...), dim3 grid, int threads, size_
     cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
 }
 
+// Split scratch per segment and sequence batch: incoming state, N_seg (fp32 [d_k, d_v] each) and the two
+// bf16 images of M_seg^T, per head.
+static size_t split_scratch_bytes(int B, int H, int d_k, int d_v, int nseg) {
+    return (size_t)nseg * B * H * (2 * (size_t)d_k * d_v * sizeof(float) + CMB_IMG);
+}
+static size_t items_bytes_aligned(uint64_t tokens, int B, int H) {
+    const size_t slots = (size_t)(tokens >> 6) + (size_t)B;
+    return (slots * H * ITEM_BYTES + 255) & ~(size_t)255;
+}
+// A split is planned only when 2 * chains <= #SMs; scratch for it is reserved for any GPU of up to this many SMs.
+constexpr int kMaxSmsForSplit = 256;
+
 size_t lean_workspace_bytes(int B, int T, int H, int d_k, int d_v, bool packed) {
     if (!tc_supported(d_k, d_v) || B <= 0 || T < 0 || H <= 0) return 0;
-    const size_t tokens = packed ? (size_t)T : (size_t)B * T;
-    const size_t slots = (tokens >> 6) + (size_t)B;
-    size_t bytes = kWorkspaceHeader + slots * H * ITEM_BYTES;
-    bytes = (bytes + 255) & ~(size_t)255;
+    const uint64_t tokens = packed ? (uint64_t)T : (uint64_t)B * T;
+    size_t bytes = kWorkspaceHeader + items_bytes_aligned(tokens, B, H);
     if (!packed) {
-        // split scratch, sized for the largest plan: incoming states, N_seg and M_seg^T per segment
-        const size_t per_seg = (size_t)B * H * d_k * (2 * (size_t)d_v + d_k) * sizeof(float);
         const size_t chains = (size_t)B * H * (d_v / DVB);
-        if (chains * 2 <= 160) bytes += kMaxSeg * per_seg;
+        if (chains * 2 <= (size_t)kMaxSmsForSplit) bytes += split_scratch_bytes(B, H, d_k, d_v, kMaxSeg);
     }
     return bytes;
+}
+
+// Set-up done once per device: the SM count and the kernels' dynamic shared-memory limits.
+constexpr int kMaxDevices = 64;
+static int device_setup(int* sms_out) {
+    static std::mutex mu;
+    static int sms_of_device[kMaxDevices] = {0};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return GDN_ERR_CUDA;
+    if (dev < 0 || dev >= kMaxDevices) return GDN_ERR_UNSUPPORTED;
+    std::lock_guard<std::mutex> lock(mu);
+    if (sms_of_device[dev] == 0) {
+        int sms = 0;
+        if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) return GDN_ERR_CUDA;
+        if (cudaFuncSetAttribute(gdn_prep_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)PREP_SMEM) != cudaSuccess ||
+            cudaFuncSetAttribute(gdn_prep_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)PREP_SMEM) != cudaSuccess ||
+            cudaFuncSetAttribute(gdn_chain_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)CHAIN_SMEM) != cudaSuccess ||
+            cudaFuncSetAttribute(gdn_chain_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)CHAIN_SMEM) != cudaSuccess ||
+            cudaFuncSetAttribute(gdn_summary_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SUM_SMEM) != cudaSuccess ||
+            cudaFuncSetAttribute(gdn_combine_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)CMB_SMEM) != cudaSuccess ||
+            cudaFuncSetAttribute(gdn_scan_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SCAN_SMEM) != cudaSuccess ||
+            cudaFuncSetAttribute(gdn_scan_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SCAN_SMEM) != cudaSuccess)
+            return GDN_ERR_CUDA;
+        sms_of_device[dev] = sms;
+    }
+    *sms_out = sms_of_device[dev];
+    return GDN_OK;
 }
 
 int launch_lean(const PrefillArgs& a, void* workspace, size_t workspace_bytes, cudaStream_t stream,
@@ -1371,25 +1723,31 @@ int launch_lean(const PrefillArgs& a, void* workspace, size_t workspace_bytes, c
     if (a.H > 65535 || a.B > 4095) return GDN_ERR_UNSUPPORTED;
     const bool packed = a.cu_seqlens != nullptr;
     const uint64_t tokens = packed ? (uint64_t)a.T : (uint64_t)a.B * a.T;
-    const size_t need = lean_workspace_bytes(a.B, a.T, a.H, a.d_k, a.d_v, packed);
-    if (!workspace || workspace_bytes < need || (reinterpret_cast<uintptr_t>(workspace) & 255u)) return GDN_ERR_WORKSPACE;
+    const size_t items_bytes = items_bytes_aligned(tokens, a.B, a.H);
+    if (!workspace || workspace_bytes < kWorkspaceHeader + items_bytes || (reinterpret_cast<uintptr_t>(workspace) & 255u))
+        return GDN_ERR_WORKSPACE;
+    int num_sms = 0;
+    if (int rc = device_setup(&num_sms)) return rc;
+    // ---- optional sequence split: planned here, before anything is launched, so that scratch that is too
+    //      small is reported (forced plan) or avoided (automatic plan) instead of being overrun ----
+    int nseg = 1, seg_chunks = 1;
+    plan_split(a.B, a.T, a.H, a.d_v, packed, num_sms, &nseg, &seg_chunks);
+    const bool forced = g_lean_force_nseg > 0 && !packed;
+    if (forced) {                                     // tests: force a segment count
+        const int nch = (a.T + C - 1) / C;
+        nseg = g_lean_force_nseg > kMaxSeg ? kMaxSeg : g_lean_force_nseg;
+        if (nseg > nch) nseg = nch > 0 ? nch : 1;
+        seg_chunks = nch > 0 ? (nch + nseg - 1) / nseg : 1;
+        nseg = nch > 0 ? (nch + seg_chunks - 1) / seg_chunks : 1;
+    }
+    if (nseg > 1 && kWorkspaceHeader + items_bytes + split_scratch_bytes(a.B, a.H, a.d_k, a.d_v, nseg) > workspace_bytes) {
+        if (forced) return GDN_ERR_WORKSPACE;
+        nseg = 1;
+        seg_chunks = (a.T + C - 1) / C > 0 ? (a.T + C - 1) / C : 1;
+    }
     CUtensorMap mq, mk, mv;
     if (!tc_make_map(&mq, a.q, tokens, a.H, a.d_k) || !tc_make_map(&mk, a.k, tokens, a.H, a.d_k) ||
         !tc_make_map(&mv, a.v, tokens, a.H, a.d_v))
-        return GDN_ERR_CUDA;
-    static int num_sms = 0;
-    if (num_sms == 0) {
-        int dev = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess ||
-            cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
-            return GDN_ERR_CUDA;
-    }
-    if (cudaFuncSetAttribute(gdn_prep_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)PREP_SMEM) != cudaSuccess ||
-        cudaFuncSetAttribute(gdn_prep_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)PREP_SMEM) != cudaSuccess ||
-        cudaFuncSetAttribute(gdn_chain_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)CHAIN_SMEM) != cudaSuccess ||
-        cudaFuncSetAttribute(gdn_chain_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)CHAIN_SMEM) != cudaSuccess ||
-        cudaFuncSetAttribute(gdn_summary_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SUM_SMEM) != cudaSuccess ||
-        cudaFuncSetAttribute(gdn_combine_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)CMB_SMEM) != cudaSuccess)
         return GDN_ERR_CUDA;
     int* ticket = static_cast<int*>(workspace);                      // header, zeroed by lean_init_workspace
     uint8_t* ws = static_cast<uint8_t*>(workspace) + kWorkspaceHeader;
@@ -1405,41 +1763,47 @@ int launch_lean(const PrefillArgs& a, void* workspace, size_t workspace_bytes, c
     count_launch();
     if (cudaGetLastError() != cudaSuccess) return GDN_ERR_CUDA;
     mark(1);
-    // ---- optional sequence split ----
-    int nseg = 1, seg_chunks = 1;
-    plan_split(a.B, a.T, a.H, a.d_v, packed, num_sms, &nseg, &seg_chunks);
-    if (g_lean_force_nseg > 0 && !packed) {           // tests: force a segment count
-        const int nch = (a.T + C - 1) / C;
-        nseg = g_lean_force_nseg > kMaxSeg ? kMaxSeg : g_lean_force_nseg;
-        if (nseg > nch) nseg = nch > 0 ? nch : 1;
-        seg_chunks = nch > 0 ? (nch + nseg - 1) / nseg : 1;
-        nseg = nch > 0 ? (nch + seg_chunks - 1) / seg_chunks : 1;
-    }
+    // ---- sequence split: segment summaries, their combination, per-segment chains ----
     float* seg_sin = nullptr;
+    g_lean_split_last = nseg > 1;
+    g_lean_scan_last = false;
+    const int nsnap = snaps ? (a.T / C) / snap_every : 0;
     if (nseg > 1) {
-        const size_t items_bytes = ((size_t)nitems * ITEM_BYTES + 255) & ~(size_t)255;
         const size_t state_elems = (size_t)a.B * nseg * a.H * a.d_k * a.d_v;
         seg_sin = reinterpret_cast<float*>(ws + items_bytes);
         float* seg_n = seg_sin + state_elems;
         float* seg_mt = seg_n + state_elems;
         SummaryParams sp{a.cu_seqlens, ws, seg_n, seg_mt, a.B, a.T, a.H, a.d_v, nseg, seg_chunks};
+        CombineParams cb{a.initial_state, seg_n, seg_mt, seg_sin, a.H, a.d_v, nseg};
+        // one resident CTA per (sequence, head, segment) runs all three phases when the grid fits the GPU at once
+        if (g_lean_use_scan && a.d_v == DVB && (long)a.B * a.H * nseg <= num_sms && (long)a.B * a.H <= kMaxScanChains) {
+            ChainParams cp{a.initial_state, static_cast<__nv_bfloat16*>(a.out), a.final_state, a.cu_seqlens,
+                           ws, seg_sin, g_lean_dbg, g_lean_drop_chunk, a.B, a.T, a.H, a.d_v, nseg, seg_chunks,
+                           snaps, snap_every, nsnap};
+            ScanParams scp{sp, cb, cp, static_cast<int*>(workspace) + kScanFlagOffset};
+            dim3 grid(1, a.H, a.B * nseg);
+            if (g_lean_dbg) launch_after(gdn_scan_kernel<true>, grid, SCAN_THREADS, SCAN_SMEM, stream, mq, mk, mv, scp);
+            else launch_after(gdn_scan_kernel<false>, grid, SCAN_THREADS, SCAN_SMEM, stream, mq, mk, mv, scp);
+            count_launch();
+            g_lean_scan_last = true;
+            mark(4);
+            return cudaGetLastError() == cudaSuccess ? GDN_OK : GDN_ERR_CUDA;
+        }
         dim3 sgrid(a.d_v / DVB, a.H, a.B * (nseg - 1));
         launch_after(gdn_summary_kernel, sgrid, SUM_THREADS, SUM_SMEM, stream, mk, mv, sp);
         count_launch();
         if (cudaGetLastError() != cudaSuccess) return GDN_ERR_CUDA;
         mark(2);
-        CombineParams cb{a.initial_state, seg_n, seg_mt, seg_sin, a.H, a.d_v, nseg};
         dim3 cgrid(a.d_v / CMB_COLS, a.H, a.B);
         launch_after(gdn_combine_kernel, cgrid, CMB_THREADS, CMB_SMEM, stream, cb);
         count_launch();
         if (cudaGetLastError() != cudaSuccess) return GDN_ERR_CUDA;
         mark(3);
     }
-    g_lean_split_last = nseg > 1;
     // ---- steps c, d ----
     ChainParams cp{a.initial_state, static_cast<__nv_bfloat16*>(a.out), a.final_state, a.cu_seqlens,
                    ws, seg_sin, g_lean_dbg, g_lean_drop_chunk, a.B, a.T, a.H, a.d_v, nseg, seg_chunks,
-                   snaps, snap_every, snaps ? (a.T / C) / snap_every : 0};
+                   snaps, snap_every, nsnap};
     dim3 grid(a.d_v / DVB, a.H, a.B * nseg);
     if (g_lean_dbg) launch_after(gdn_chain_kernel<true>, grid, CHAIN_THREADS, CHAIN_SMEM, stream, mq, mk, mv, cp);
     else launch_after(gdn_chain_kernel<false>, grid, CHAIN_THREADS, CHAIN_SMEM, stream, mq, mk, mv, cp);
@@ -1448,6 +1812,7 @@ int launch_lean(const PrefillArgs& a, void* workspace, size_t workspace_bytes, c
     return cudaGetLastError() == cudaSuccess ? GDN_OK : GDN_ERR_CUDA;
 }
 
+void lean_set_scan(int enable) { g_lean_use_scan = enable != 0; }
 void lean_force_segments(int nseg) { g_lean_force_nseg = nseg; }
 void lean_set_debug(float* p) { g_lean_dbg = p; }
 void lean_set_drop_chunk(int c) { g_lean_drop_chunk = c; }
@@ -1464,18 +1829,20 @@ int lean_set_timing(int enable) {
     return GDN_OK;
 }
 
-// milliseconds of {prepare, summary, combine, chain} of the most recent call (0 for kernels not run)
-int lean_get_timing(float* ms4) {
-    for (int i = 0; i < 4; ++i) ms4[i] = 0.f;
+// milliseconds of {prepare, summary, combine, chain, scan} of the most recent call (0 for kernels not run)
+int lean_get_timing(float* ms5) {
+    for (int i = 0; i < 5; ++i) ms5[i] = 0.f;
     if (!g_lean_events[0]) return GDN_ERR_INVALID_ARG;
     if (cudaEventSynchronize(g_lean_events[4]) != cudaSuccess) return GDN_ERR_CUDA;
-    bool ok = cudaEventElapsedTime(&ms4[0], g_lean_events[0], g_lean_events[1]) == cudaSuccess;
-    if (g_lean_split_last) {
-        ok = ok && cudaEventElapsedTime(&ms4[1], g_lean_events[1], g_lean_events[2]) == cudaSuccess;
-        ok = ok && cudaEventElapsedTime(&ms4[2], g_lean_events[2], g_lean_events[3]) == cudaSuccess;
-        ok = ok && cudaEventElapsedTime(&ms4[3], g_lean_events[3], g_lean_events[4]) == cudaSuccess;
+    bool ok = cudaEventElapsedTime(&ms5[0], g_lean_events[0], g_lean_events[1]) == cudaSuccess;
+    if (g_lean_scan_last) {
+        ok = ok && cudaEventElapsedTime(&ms5[4], g_lean_events[1], g_lean_events[4]) == cudaSuccess;
+    } else if (g_lean_split_last) {
+        ok = ok && cudaEventElapsedTime(&ms5[1], g_lean_events[1], g_lean_events[2]) == cudaSuccess;
+        ok = ok && cudaEventElapsedTime(&ms5[2], g_lean_events[2], g_lean_events[3]) == cudaSuccess;
+        ok = ok && cudaEventElapsedTime(&ms5[3], g_lean_events[3], g_lean_events[4]) == cudaSuccess;
     } else {
-        ok = ok && cudaEventElapsedTime(&ms4[3], g_lean_events[1], g_lean_events[4]) == cudaSuccess;
+        ok = ok && cudaEventElapsedTime(&ms5[3], g_lean_events[1], g_lean_events[4]) == cudaSuccess;
     }
     return ok ? GDN_OK : GDN_ERR_CUDA;
 }
@@ -1500,7 +1867,6 @@ int lean_get_timing(float* ms4) {
 constexpr size_t kStaticScratchBytes = 64ull << 20;            // 64 MiB
 static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
 static __device__ int g_static_ticket[2];                      // the prepare kernel's item ticket (zero at load)
-constexpr int kMaxDevices = 64;
 
 int launch_lean_static(const PrefillArgs& a, cudaStream_t stream) {
     if (!tc_supported(a.d_k, a.d_v)) return GDN_ERR_UNSUPPORTED;

@@ -105,3 +105,31 @@ def test_packed_sequences_are_independent():
     np.testing.assert_allclose(packed[7:], oracle.attention_causal(q[:, 7:], k[:, 7:], v[:, 7:], 0.4)[0], rtol=1e-14)
     # first token of every sequence returns its own value: nothing leaks across the boundary
     np.testing.assert_allclose(packed[7, 0], v[0, 7, 0], rtol=1e-14)
+
+
+def test_rows_variant_against_full_definition_and_scalar_brute_force():
+    """attention_causal_rows (the sampled-row form the full-size GPU checks use) on every row of a small
+    grouped-query case: equal to attention_causal, and to scalar loops that know nothing of numpy.  A slip
+    in its head grouping or in its prefix length fails here, on the CPU."""
+    rng = np.random.default_rng(7)
+    q, k, v = _rand(rng, B=2, T=9, Hq=6, Hkv=2, d=4)      # three query heads per key/value head
+    scale = 0.4
+    rows = [(b, i, h) for b in range(2) for i in range(9) for h in range(6)]
+    got = oracle.attention_causal_rows(q, k, v, scale, rows)
+    full = oracle.attention_causal(q, k, v, scale)
+    for n, (b, i, h) in enumerate(rows):
+        np.testing.assert_allclose(got[n], full[b, i, h], rtol=1e-13, atol=1e-15)
+    for n, (b, i, h) in enumerate(rows[::7]):
+        hk = h // 3
+        den, num = 0.0, [0.0] * 4
+        for j in range(i + 1):
+            w = math.exp(sum(q[b, i, h, f] * k[b, j, hk, f] for f in range(4)) * scale)
+            den += w
+            for f in range(4):
+                num[f] += w * v[b, j, hk, f]
+        np.testing.assert_allclose(got[7 * n], [x / den for x in num], rtol=1e-12)
+    # an out-of-order, repeated selection returns the rows in the order asked for
+    pick = [(1, 8, 5), (0, 0, 0), (1, 8, 5), (0, 4, 3)]
+    sub = oracle.attention_causal_rows(q, k, v, scale, pick)
+    for n, (b, i, h) in enumerate(pick):
+        np.testing.assert_allclose(sub[n], full[b, i, h], rtol=1e-13, atol=1e-15)

@@ -5,7 +5,7 @@ import pytest
 import torch
 
 import paper_2607_14568_b200 as gdn
-from workloads import chain_inputs, get_config, make_inputs, widen
+from workloads import bf16_bits_to_f32, f32_to_bf16_bits, get_config, make_inputs, widen
 
 import oracle
 from gdn_testlib import (BF16_MAX_ABS, BF16_REL_L2, F32_REL_L2, assert_close, f64, prefill_fused,
@@ -114,19 +114,24 @@ def test_bf16_packed_ragged(impl):
         assert torch.equal(o1[0], out[a:b]) and torch.equal(f1[0], fin[n])
 
 
+@pytest.mark.parametrize("merged", [1, 0])
 @pytest.mark.parametrize("T,nseg,gate", [(640, 2, 0.05), (1000, 3, 0.05), (2048, 5, 0.001), (4096, 16, 0.0),
-                                         (333, 4, 0.02)])
-def test_two_kernel_sequence_split(T, nseg, gate):
-    """The sequence split (segment summaries M, N; fp32 combination; per-segment chains) against the
+                                         (333, 4, 0.02), (3000, 9, 0.0)])
+def test_two_kernel_sequence_split(T, nseg, gate, merged):
+    """The sequence split (segment summaries M, N; their combination; per-segment chains) against the
     oracle, including weak or no decay, where a segment's outgoing state depends fully on its
-    incoming one."""
+    incoming one.  merged = 1: the three phases in one launch (CTAs hand over through counters in global
+    memory); merged = 0: three kernels."""
     cfg = get_config("long", T=T, H=2, gate_scale=gate, seed=60 + nseg)
     x = make_inputs(cfg)
     gdn.lib().gdn_debug_force_segments(nseg)
+    gdn.lib().gdn_debug_set_scan(merged)
     try:
-        check_bf16(x, prefill_two_kernel, f"split T={T} nseg={nseg}")
+        check_bf16(x, prefill_two_kernel, f"split T={T} nseg={nseg} merged={merged}")
+        check_bf16(x, prefill_two_kernel, f"split T={T} nseg={nseg} merged={merged}, second call")   # counters were left clean
     finally:
         gdn.lib().gdn_debug_force_segments(0)
+        gdn.lib().gdn_debug_set_scan(1)
 
 
 def test_two_kernel_sequence_split_wide_values_and_batch():
@@ -171,25 +176,88 @@ def test_bf16_full_configs(name, impl):
     print(f"\n{name}/{impl}: out rel-L2 {ro:.2e} max-abs {mo:.2e}; state rel-L2 {rs:.2e} max-abs {ms:.2e}")
 
 
+_LARGE_ORACLE = {}
+
+
+def _large_oracle(cfg, x):
+    """fp64 recurrence over every (sequence, head) chain of `large`, 16 heads of one sequence at a time
+    (the oracle runs one chain per host thread); computed once per test session."""
+    if not _LARGE_ORACLE:
+        for n in range(cfg.B):
+            for h0 in range(0, cfg.H, 16):
+                hs = slice(h0, min(cfg.H, h0 + 16))
+                o_ref, f_ref = oracle.sequential(widen(x.q[n:n + 1, :, hs]), widen(x.k[n:n + 1, :, hs]),
+                                                 widen(x.v[n:n + 1, :, hs]), x.log_alpha[n:n + 1, :, hs],
+                                                 x.beta[n:n + 1, :, hs], None)
+                _LARGE_ORACLE[(n, h0)] = (o_ref[0].astype(np.float32), f_ref[0])
+    return _LARGE_ORACLE
+
+
 @pytest.mark.parametrize("impl", ["fused", "two_kernel"])
-def test_bf16_large_sampled_chains(impl):
-    """Configuration 'large' (B=4, T=32768, H=32, d_v=256) at full size; the oracle checks a seeded
-    sample of whole (sequence, head) chains (heads are independent, so each checked chain is
-    checked completely) and every other chain is checked for finiteness."""
+def test_bf16_large_all_chains(impl):
+    """Configuration 'large' (B=4, T=32768, H=32, d_v=256) at full size: every one of the 128 (sequence, head)
+    chains is compared with the fp64 recurrence, outputs and final state (the reference outputs are kept in
+    fp32, eight decimal digits, far below the bf16 tolerances)."""
     cfg = get_config("large")
     x = make_inputs(cfg, threads=16)
     d = to_device(x)
     out, fin = run_lib(BF16_FNS[impl], d)
     assert bool(torch.isfinite(out).all()) and bool(torch.isfinite(fin).all())
-    rng = np.random.default_rng(5)
-    chains = {(0, 0), (cfg.B - 1, cfg.H - 1)} | {(int(rng.integers(cfg.B)), int(rng.integers(cfg.H))) for _ in range(4)}
-    for n, h in sorted(chains):
-        c = chain_inputs(cfg, n, h)
-        o_ref, f_ref = oracle.sequential(widen(c["q"])[None, :, None], widen(c["k"])[None, :, None],
-                                         widen(c["v"])[None, :, None], c["log_alpha"][None, :, None],
-                                         c["beta"][None, :, None], None)
-        assert_close(f64(out[n, :, h]), o_ref[0, :, 0], BF16_REL_L2, BF16_MAX_ABS, f"large chain {(n, h)} out")
-        assert_close(f64(fin[n, h]), f_ref[0, 0], BF16_REL_L2, BF16_MAX_ABS, f"large chain {(n, h)} state")
+    ref = _large_oracle(cfg, x)
+    worst = 0.0
+    for (n, h0), (o_ref, f_ref) in sorted(ref.items()):
+        hs = slice(h0, h0 + o_ref.shape[1])
+        r, _ = assert_close(f64(out[n, :, hs]), o_ref.astype(np.float64), BF16_REL_L2, BF16_MAX_ABS,
+                            f"large seq {n} heads {h0}.. out")
+        assert_close(f64(fin[n, hs]), f_ref, BF16_REL_L2, BF16_MAX_ABS, f"large seq {n} heads {h0}.. state")
+        worst = max(worst, r)
+    print(f"\nlarge/{impl}: worst out rel-L2 over head groups {worst:.2e}")
+
+
+# ---- final_state written over initial_state ------------------------------------------------------------
+@pytest.mark.parametrize("impl,nseg,H", [("fused", 0, 4), ("two_kernel", 0, 4), ("two_kernel", 3, 64),
+                                         ("two_kernel", 16, 16), ("two_kernel", 9, 16)])
+def test_bf16_final_state_may_alias_initial_state(impl, nseg, H):
+    """The header allows final_state == initial_state.  With the sequence split the grid of the last kernel
+    (H * nseg CTAs: 192 and 256 in two of the cases) does not fit the GPU in one wave, so a segment-0 CTA may well
+    start after a last-segment CTA has finished; 16 heads x 9 segments run as the merged single launch.  The result
+    must still be the recurrence from the given initial state."""
+    cfg = get_config("long", T=1088, H=H, init_std=0.5, seed=90 + nseg)
+    x = make_inputs(cfg)
+    d = to_device(x)
+    d["final_state"] = d["initial_state"]
+    gdn.lib().gdn_debug_force_segments(nseg)
+    try:
+        out, fin = run_lib(BF16_FNS[impl], d)
+    finally:
+        gdn.lib().gdn_debug_force_segments(0)
+    o_ref, f_ref = run_oracle(x)
+    assert_close(f64(out), o_ref, BF16_REL_L2, BF16_MAX_ABS, "aliased out")
+    assert_close(f64(fin), f_ref, BF16_REL_L2, BF16_MAX_ABS, "aliased final_state")
+
+
+# ---- inputs outside the usual ranges: computed as given, no clamping -----------------------------------------
+@pytest.mark.parametrize("impl", ["fused", "two_kernel", "simt"])
+@pytest.mark.parametrize("case", ["beta_0_1_1p5", "growing_gates", "key_norm_half", "key_norm_1p5"])
+def test_bf16_unclamped_inputs(impl, case):
+    """beta outside (0, 1), a few positive log gates, keys that are not unit vectors: the library applies no
+    clamp and no check, so the result is still the recurrence on the values given.  Keys of norm 1.5 with
+    beta near 1 make I - beta k k^T expansive (|1 - 2.25 beta| > 1); the inputs are sized so that fp64 itself
+    stays bounded, and the bf16 path must stay within its usual tolerance of it."""
+    cfg = get_config("long", T=300, H=2, init_std=0.02, seed=95)
+    x = make_inputs(cfg)
+    rng = np.random.default_rng(96)
+    if case == "beta_0_1_1p5":
+        x.beta[...] = rng.choice(np.array([0.0, 1.0, 1.5], dtype=np.float32), size=x.beta.shape, p=[0.3, 0.5, 0.2])
+    elif case == "growing_gates":
+        idx = rng.random(x.log_alpha.shape) < 0.05
+        x.log_alpha[idx] = 0.03                                   # alpha > 1 on one token in twenty
+    else:
+        s = 0.5 if case == "key_norm_half" else 1.5
+        x.k[...] = f32_to_bf16_bits(bf16_bits_to_f32(x.k) * np.float32(s))
+        if s > 1:
+            x.beta[...] *= 0.4                                    # keeps |1 - beta |k|^2| below one
+    check_bf16(x, BF16_FNS[impl], f"{impl} {case}")
 
 
 # ---- host-buffer entry point ------------------------------------------------------------------------
@@ -205,7 +273,10 @@ def test_host_entry_matches_device_entry():
     o2, f2 = gdn.gdn_chunk_prefill_host(h["q"], h["k"], h["v"], h["log_alpha"], h["beta"], h["initial_state"],
                                         h["out"], h["final_state"], h["cu_seqlens"], staging)
     torch.cuda.synchronize()
-    assert torch.equal(o2, out.cpu()) and torch.equal(f2, fin.cpu())
+    o_ref, f_ref = run_oracle(x)
+    assert_close(f64(o2), o_ref, BF16_REL_L2, BF16_MAX_ABS, "host entry out vs oracle")
+    assert_close(f64(f2), f_ref, BF16_REL_L2, BF16_MAX_ABS, "host entry final_state vs oracle")
+    assert torch.equal(o2, out.cpu()) and torch.equal(f2, fin.cpu())      # and bit for bit the device entry point
     with pytest.raises(gdn.GdnError) as e:
         gdn.gdn_chunk_prefill_host(h["q"], h["k"], h["v"], h["log_alpha"], h["beta"], h["initial_state"],
                                    h["out"], h["final_state"], h["cu_seqlens"], staging[:1024])
