@@ -135,7 +135,7 @@ size_t gdn_host_staging_bytes(int B, int T, int H, int d_k, int d_v);
 
 /*
  * One decode step: the same recurrence for a single new token per sequence, continuing from
- * the state a prefill returned (Section "The model": the state is "updated token-by-token";
+ * the state a prefill returned (Section "The model": the state advances by one token at a time;
  * Section "Decode, and why 4-bit is slower": decode is bandwidth-bound -- here the state is
  * read once and written once).  q, k [B, H, d_k] and v, out [B, H, d_v] are bf16; log_alpha,
  * beta [B, H] fp32; state [B, H, d_k, d_v] fp32 is updated IN PLACE (it is both the incoming
@@ -167,7 +167,7 @@ int gdn_chunk_prefill_snapshots(const void* q, const void* k, const void* v,
                                 gdn_stream_t stream);
 
 /*
- * gdn_chunk_prefill with the per-position prologue fused in (Section "Batched prefill": the norms
+ * gdn_chunk_prefill with the per-position prologue fused in (Section "Prefill projections: dequantize, then call the vendor": the norms
  * and gating around the projections are batched over the chunk).  q_raw, k_raw are the raw bf16
  * projections and a_raw, b_raw the fp32 gate pre-activations, same shapes as q, k, log_alpha, beta
  * of gdn_chunk_prefill.  The call computes, per (token, head),
@@ -195,13 +195,15 @@ int gdn_chunk_prefill_raw(const void* q_raw, const void* k_raw, const void* v,
  * which each (sequence, head) chain also does its own forward substitutions.  With scratch of
  * at least gdn_workspace_bytes(...) bytes the state-independent steps (cumulative gate,
  * token-token matrices, forward substitution, WY factor W) run first as a kernel over every
- * (chunk, head) on all SMs -- "all C positions are solved together", Section "A chunked
+ * (chunk, head) on all SMs -- every position of a chunk is resolved at once, Section "A chunked
  * delta-rule scan for the recurrent layers" -- and leave their results in the scratch for the
  * chain kernel; this is the faster path.  The scratch stays owned by the caller, is 256-byte
  * aligned device memory, must outlive every call that uses it, and is shared by all calls
- * (calls on different streams must not overlap).  gdn_set_workspace zeroes the first 256 bytes
- * with a synchronous cudaMemset (a work counter that every call leaves at zero again; the caller
- * must not write there between calls) and returns GDN_ERR_CUDA if that fails; a pointer that is
+ * (calls on different streams must not overlap).  The scratch belongs to the device that is current
+ * when gdn_set_workspace is called: every device has its own, and a call uses the one of the device
+ * current at that call.  gdn_set_workspace zeroes the first 4096 bytes with a synchronous cudaMemset
+ * (work counters that every call leaves at zero again; the caller must not write there between calls;
+ * after a call that reported GDN_ERR_TIMEOUT set the workspace again before reusing it) and returns GDN_ERR_CUDA if that fails; a pointer that is
  * not 256-byte aligned gives GDN_ERR_UNSUPPORTED.  gdn_set_workspace(NULL, 0) removes it.
  * `packed` is 1 when cu_seqlens will be passed (T = total tokens), else 0.
  * gdn_workspace_bytes returns 0 for sizes the tensor-core path does not support.
@@ -249,6 +251,15 @@ int gdn_chunk_prefill_noalloc(const void* q, const void* k, const void* v,
  * of that call are undefined.  GDN_ERR_CUDA if the device reports an error.
  */
 int gdn_query_status(void);
+
+/*
+ * The same status, but waiting only for `stream` (cudaStreamSynchronize): everything enqueued on that
+ * stream before this call has finished when it returns, other streams of the device keep running.  The
+ * status word is shared by all streams of a device, so a time-out raised by a call on another stream that
+ * has already run shows up here too.  (Failure reporting of the bounded device-side waits; the paper's
+ * engine has no counterpart.)
+ */
+int gdn_query_status_stream(gdn_stream_t stream);
 
 /* Number of kernels this library has launched in this process so far. */
 unsigned long long gdn_launch_count(void);

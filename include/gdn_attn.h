@@ -2,7 +2,7 @@
  * gdn_attn.h -- C ABI of the causal softmax attention of the hybrid backbone's attention layers
  * (second workload of libgdn; status codes and gdn_stream_t come from gdn.h).
  *
- * The operation (Section "Batched attention": scores for all queries of a block as one matrix
+ * The operation (Sections "The layout trick" and "Prefill attention: finding and removing the O(N^2) wall": scores for all queries of a block as one matrix
  * product, a softmax that normalises only the causally valid prefix and leaves exact zeros after
  * it, a second product with V; grouped-query attention by letting several query heads address
  * the same key/value block).  For every sequence b, query head h and position i:

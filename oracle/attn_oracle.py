@@ -1,7 +1,7 @@
 """fp64 CPU oracle for causal softmax attention with grouped queries (test infrastructure only).
 
-Section "Batched attention" of the paper rewrites the prefill attention of the softmax layers as
-per-head matrix products: scores S = Q K^T for the whole chunk, a column softmax that normalises
+Sections "The layout trick" and "Prefill attention: finding and removing the O(N^2) wall" of the
+paper rewrite the prefill attention of the softmax layers as per-head matrix products: scores S = Q K^T for the whole chunk, a column softmax that normalises
 only the causally valid prefix and zeroes the tail, then a second product with V; several query
 heads share one key/value head by addressing the same K/V block.
 

@@ -23,6 +23,13 @@
 //   gdn_oracle_dense       brute force: the whole sequence as one T x T system
 //                          solved by general Gaussian elimination with pivoting
 //                          (it does not know the matrix is triangular).
+//   gdn_oracle_chunked_stages  gdn_oracle_chunked (form 0) for ONE (sequence, head)
+//                          chain that also hands out what it computes on the way,
+//                          chunk by chunk: g, A, P, T, W, U, Delta and the state each
+//                          chunk starts from -- so that a GPU path can be compared
+//                          stage by stage, each stage with its own reference (Section
+//                          "Porting the Vision Tower, Stage by Stage").  Same code,
+//                          same arithmetic; the extra outputs are copies.
 //
 // Pins (tests/test_oracle_pins.py): every function here is pinned by closed
 // forms and invariants (pure decay, exact key overwrite, one-token closed form,
@@ -119,7 +126,14 @@ void sequential_chain(const Problem& p, int n, int h) {
 //   O   = diag(e^{g}) Q S0 + P Delta
 // A tail chunk simply has fewer rows.
 // ---------------------------------------------------------------------------
-void chunked_chain(const Problem& p, int n, int h, int C, int form) {
+// Optional per-chunk copies of the intermediates of chunked_chain (any pointer may be null).
+// Layouts, ci = chunk index: g [ci][C]; A, P, T [ci][C][C]; W [ci][C][dk]; U, D [ci][C][dv];
+// Sin [ci][dk][dv].  Rows beyond a tail chunk's length are left untouched.
+struct Stages {
+    double *g, *A, *P, *T, *W, *U, *D, *Sin;
+};
+
+void chunked_chain(const Problem& p, int n, int h, int C, int form, const Stages* st = nullptr) {
     const int dk = p.dk, dv = p.dv, H = p.H;
     long tok0; int len; seq_range(p, n, tok0, len);
     std::vector<double> S((size_t)dk * dv, 0.0), Snew((size_t)dk * dv);
@@ -130,6 +144,8 @@ void chunked_chain(const Problem& p, int n, int h, int C, int form) {
 
     for (int c0 = 0; c0 < len; c0 += C) {
         const int R = std::min(C, len - c0);
+        const size_t ci = (size_t)(c0 / C);
+        if (st && st->Sin) std::memcpy(st->Sin + ci * dk * dv, S.data(), sizeof(double) * dk * dv);
         auto K = [&](int r) { return p.k + ((size_t)(tok0 + c0 + r) * H + h) * dk; };
         auto Q = [&](int r) { return p.q + ((size_t)(tok0 + c0 + r) * H + h) * dk; };
         auto V = [&](int r) { return p.v + ((size_t)(tok0 + c0 + r) * H + h) * dv; };
@@ -165,6 +181,16 @@ void chunked_chain(const Problem& p, int n, int h, int C, int form) {
                 U[(size_t)r * dv + j] = x;
             }
         }
+        if (st) {
+            for (int r = 0; r < R; ++r) {
+                if (st->g) st->g[ci * C + r] = g[r];
+                if (st->A) std::memcpy(st->A + (ci * C + r) * C, &A[(size_t)r * C], sizeof(double) * R);
+                if (st->P) std::memcpy(st->P + (ci * C + r) * C, &P[(size_t)r * C], sizeof(double) * R);
+                if (st->T) std::memcpy(st->T + (ci * C + r) * C, &Tm[(size_t)r * C], sizeof(double) * R);
+                if (st->W) std::memcpy(st->W + (ci * C + r) * dk, &W[(size_t)r * dk], sizeof(double) * dk);
+                if (st->U) std::memcpy(st->U + (ci * C + r) * dv, &U[(size_t)r * dv], sizeof(double) * dv);
+            }
+        }
         const double gC = g[R - 1];
         if (form == 0) {
             // correction Delta = U - W S0, output, state
@@ -174,6 +200,8 @@ void chunked_chain(const Problem& p, int n, int h, int C, int form) {
                     for (int m = 0; m < dk; ++m) x -= W[(size_t)r * dk + m] * S[(size_t)m * dv + j];
                     D[(size_t)r * dv + j] = x;
                 }
+            if (st && st->D)
+                for (int r = 0; r < R; ++r) std::memcpy(st->D + (ci * C + r) * dv, &D[(size_t)r * dv], sizeof(double) * dv);
             for (int r = 0; r < R; ++r) {
                 double* o = p.out + ((size_t)(tok0 + c0 + r) * H + h) * dv;
                 for (int j = 0; j < dv; ++j) {
@@ -356,6 +384,22 @@ int gdn_oracle_chunked(const double* q, const double* k, const double* v,
     const int chains = B * H;
 #pragma omp parallel for schedule(dynamic, 1)
     for (int c = 0; c < chains; ++c) chunked_chain(p, c / H, c % H, chunk, form);
+    return 0;
+}
+
+// One chain (sequence n, head h), form 0, with the per-chunk intermediates copied out.  out and final_state
+// are written for that chain only (same layouts as above; other chains' entries are left untouched).
+int gdn_oracle_chunked_stages(const double* q, const double* k, const double* v,
+                              const double* log_alpha, const double* beta,
+                              const double* initial_state, double* out, double* final_state,
+                              const int32_t* cu_seqlens, int B, int T, int H, int d_k, int d_v,
+                              int chunk, int n, int h,
+                              double* g, double* A, double* P, double* Tm, double* W, double* U, double* D,
+                              double* Sin) {
+    Problem p{q, k, v, log_alpha, beta, initial_state, out, final_state, cu_seqlens, B, T, H, d_k, d_v};
+    if (!valid(p) || chunk <= 0 || n < 0 || n >= B || h < 0 || h >= H) return 1;
+    const Stages st{g, A, P, Tm, W, U, D, Sin};
+    chunked_chain(p, n, h, chunk, 0, &st);
     return 0;
 }
 

@@ -11,7 +11,10 @@ the C file: ``q,k [B,T,H,d_k]``, ``v [B,T,H,d_v]``, ``log_alpha,beta [B,T,H]``,
   chunked     the intra-/inter-chunk form of the same section (form=1: its
               S' = M S + N variant)
   dense       the whole sequence as one general linear system (brute force)
-  prologue    the per-position kernels in front of the scan (Section "Batched prefill":
+  chunked_stages  the chunked form for one (sequence, head) chain, also returning its per-chunk
+              intermediates (g, A, P, T, W, U, Delta, incoming state): stage-by-stage references in the
+              sense of Section "Porting the Vision Tower, Stage by Stage"
+  prologue    the per-position kernels in front of the scan (Section "Prefill projections: dequantize, then call the vendor":
               norms and gating batched over the chunk): L2 norm of q and k over the feature
               axis, beta = sigmoid(b), log_alpha = -softplus(a) * gate_scale.  The paper names
               these kernels without printing formulas; the forms here are the reading the
@@ -38,8 +41,9 @@ def _load():
         lib.gdn_oracle_sequential.argtypes = common
         lib.gdn_oracle_dense.argtypes = common
         lib.gdn_oracle_chunked.argtypes = common + [ctypes.c_int, ctypes.c_int]
+        lib.gdn_oracle_chunked_stages.argtypes = common + [ctypes.c_int] * 3 + [dp] * 8
         for f in (lib.gdn_oracle_sequential, lib.gdn_oracle_dense, lib.gdn_oracle_chunked,
-                  lib.gdn_oracle_num_threads):
+                  lib.gdn_oracle_chunked_stages, lib.gdn_oracle_num_threads):
             f.restype = ctypes.c_int
         _lib = lib
     return _lib
@@ -104,6 +108,28 @@ def sequential(q, k, v, log_alpha, beta, initial_state=None, cu_seqlens=None):
 def chunked(q, k, v, log_alpha, beta, initial_state=None, cu_seqlens=None, chunk=64, form=0):
     arrs, dims = _prepare(q, k, v, log_alpha, beta, initial_state, cu_seqlens)
     return _call(_load().gdn_oracle_chunked, arrs, dims, int(chunk), int(form))
+
+
+def chunked_stages(q, k, v, log_alpha, beta, initial_state=None, cu_seqlens=None, chunk=64, n=0, h=0):
+    """The chunked form (form 0) of chain (n, h) with its intermediates.  Returns a dict of fp64 arrays, nch =
+    number of chunks of the sequence: g [nch,C], A, P, T [nch,C,C], W [nch,C,d_k], U, Delta [nch,C,d_v],
+    S_in [nch,d_k,d_v] (the state each chunk starts from), out [len,d_v], final_state [d_k,d_v], length.
+    Rows beyond the length of a tail chunk are zero."""
+    arrs, dims = _prepare(q, k, v, log_alpha, beta, initial_state, cu_seqlens)
+    B, T, H, dk, dv = dims
+    cu = arrs[8]
+    length = int(cu[n + 1] - cu[n]) if cu is not None else T
+    tok0 = int(cu[n]) if cu is not None else n * T
+    C = int(chunk)
+    nch = (length + C - 1) // C
+    z = lambda *shape: np.zeros(shape, dtype=np.float64)
+    st = dict(g=z(nch, C), A=z(nch, C, C), P=z(nch, C, C), T=z(nch, C, C), W=z(nch, C, dk), U=z(nch, C, dv),
+              Delta=z(nch, C, dv), S_in=z(nch, dk, dv))
+    out, fin = _call(_load().gdn_oracle_chunked_stages, arrs, dims, C, int(n), int(h),
+                     *[_ptr(st[name]) for name in ("g", "A", "P", "T", "W", "U", "Delta", "S_in")])
+    flat = out.reshape(-1, H, dv)
+    st.update(out=flat[tok0:tok0 + length, h].copy(), final_state=fin[n, h].copy(), length=length)
+    return st
 
 
 def dense(q, k, v, log_alpha, beta, initial_state=None, cu_seqlens=None):

@@ -74,6 +74,12 @@ def lib():
         L.gdn_debug_set_scan.restype = None
         L.gdn_query_status.argtypes = []
         L.gdn_query_status.restype = i
+        L.gdn_query_status_stream.argtypes = [vp]
+        L.gdn_query_status_stream.restype = i
+        L.gdn_debug_set_l2_hints.argtypes = [i]
+        L.gdn_debug_set_l2_hints.restype = None
+        L.gdn_debug_set_chain_stamps.argtypes = [vp]
+        L.gdn_debug_set_chain_stamps.restype = None
         L.gdn_debug_set_dump.argtypes = [vp]
         L.gdn_debug_set_dump.restype = None
         L.gdn_launch_count.argtypes = []
@@ -114,6 +120,11 @@ def gdn_set_workspace(workspace: Optional[torch.Tensor]) -> None:
 def gdn_query_status() -> int:
     """Synchronises the device and returns the kernels' status word (0 = ok)."""
     return int(lib().gdn_query_status())
+
+
+def gdn_query_status_stream(stream=None) -> int:
+    """Waits for `stream` only (default: torch's current stream) and returns the kernels' status word."""
+    return int(lib().gdn_query_status_stream(_stream(stream)))
 
 
 def gdn_launch_count() -> int:

@@ -1,7 +1,7 @@
 // Causal softmax attention with grouped queries on the 5th-generation tensor core (sm_100a).
 //
-// Section "Batched attention" of the paper turns the prefill attention of the softmax layers
-// into matrix products: scores for a whole block of queries at once, a softmax that normalises
+// Sections "The layout trick" and "Prefill attention: finding and removing the O(N^2) wall" of the
+// paper turn the prefill attention of the softmax layers into matrix products: scores for a whole block of queries at once, a softmax that normalises
 // the causally valid prefix and leaves exact zeros beyond it, a second product with V, and
 // grouped queries by pointing several query heads at one key/value block.  The paper materialises
 // the score matrix in a buffer it already owned; here a tile of scores lives only in tensor
@@ -363,6 +363,11 @@ attn_causal_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
 }  // namespace
 
 bool attn_supported(int Hq, int Hkv, int d) { return d == HD && Hkv > 0 && Hq > 0 && Hq % Hkv == 0; }
+
+int attn_status_async(int* host_dst, cudaStream_t stream) {
+    return cudaMemcpyFromSymbolAsync(host_dst, g_attn_status, sizeof(int), 0, cudaMemcpyDeviceToHost, stream) == cudaSuccess
+               ? GDN_OK : GDN_ERR_CUDA;
+}
 
 int attn_query_status() {
     int st = 0;

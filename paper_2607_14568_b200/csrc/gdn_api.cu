@@ -1,6 +1,7 @@
 // C-ABI entry points of libgdn: argument validation and dispatch.  See include/gdn.h.
 
 #include <atomic>
+#include <mutex>
 #include <vector>
 
 #include "gdn_internal.h"
@@ -33,17 +34,30 @@ PrefillArgs pack(const void* q, const void* k, const void* v, const float* log_a
     return PrefillArgs{q, k, v, log_alpha, beta, initial_state, out, final_state, cu_seqlens, B, T, H, d_k, d_v};
 }
 
-// Caller-provided scratch (gdn_set_workspace) and the path override used by the tests.
-void* g_workspace = nullptr;
-size_t g_workspace_bytes = 0;
-int g_force_path = 0;   // 0 = automatic, 1 = fused kernel, 2 = two-kernel pipeline
+// Caller-provided scratch (gdn_set_workspace), one per device: a pointer is only valid on the device that was
+// current when it was set, so calls look up the scratch of the device that is current when they are made.
+constexpr int kMaxDevices = 64;
+struct Workspace {
+    void* ptr = nullptr;
+    size_t bytes = 0;
+};
+Workspace g_workspace_of_device[kMaxDevices];
+std::mutex g_workspace_mutex;
+Workspace current_workspace() {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return Workspace{};
+    std::lock_guard<std::mutex> lock(g_workspace_mutex);
+    return g_workspace_of_device[dev];
+}
+int g_force_path = 0;   // tests: 0 = automatic, 1 = fused kernel, 2 = two-kernel pipeline
 
 int dispatch_bf16(const PrefillArgs& a, cudaStream_t stream) {
     if (!tc_supported(a.d_k, a.d_v)) return launch_simt(a, /*io_bf16=*/true, stream);
     const uint64_t tokens = a.cu_seqlens ? (uint64_t)a.T : (uint64_t)a.B * a.T;
     if (tokens == 0 || g_force_path == 1) return launch_tc(a, stream);
     const size_t need = lean_workspace_bytes(a.B, a.T, a.H, a.d_k, a.d_v, a.cu_seqlens != nullptr);
-    if (g_workspace && g_workspace_bytes >= need) return launch_lean(a, g_workspace, g_workspace_bytes, stream);
+    const Workspace ws = current_workspace();
+    if (ws.ptr && ws.bytes >= need) return launch_lean(a, ws.ptr, ws.bytes, stream);
     if (g_force_path == 2) return GDN_ERR_WORKSPACE;
     return launch_tc(a, stream);
 }
@@ -267,11 +281,12 @@ int gdn_chunk_prefill_snapshots(const void* q, const void* k, const void* v, con
     if (!aligned16(snapshots) || !tc_supported(d_k, d_v)) return GDN_ERR_UNSUPPORTED;
     if (T == 0) return launch_tc(a, reinterpret_cast<cudaStream_t>(stream));
     const size_t need = lean_workspace_bytes(B, T, H, d_k, d_v, false);
-    if (!g_workspace || g_workspace_bytes < need) return GDN_ERR_WORKSPACE;
+    const Workspace ws = current_workspace();
+    if (!ws.ptr || ws.bytes < need) return GDN_ERR_WORKSPACE;
     LeanOptions opt;
     opt.snaps = snapshots;
     opt.snap_every = snapshot_every_chunks;
-    return launch_lean(a, g_workspace, g_workspace_bytes, reinterpret_cast<cudaStream_t>(stream), opt);
+    return launch_lean(a, ws.ptr, ws.bytes, reinterpret_cast<cudaStream_t>(stream), opt);
 }
 
 int gdn_chunk_prefill_raw(const void* q_raw, const void* k_raw, const void* v, const float* a_raw, const float* b_raw,
@@ -285,12 +300,13 @@ int gdn_chunk_prefill_raw(const void* q_raw, const void* k_raw, const void* v, c
     const long tokens = cu_seqlens ? (long)T : (long)B * T;
     if (tokens == 0) return launch_tc(a, reinterpret_cast<cudaStream_t>(stream));   // only copies the states
     const size_t need = lean_workspace_bytes(B, T, H, d_k, d_v, cu_seqlens != nullptr);
-    if (!g_workspace || g_workspace_bytes < need) return GDN_ERR_WORKSPACE;
+    const Workspace ws = current_workspace();
+    if (!ws.ptr || ws.bytes < need) return GDN_ERR_WORKSPACE;
     LeanOptions opt;
     opt.raw = true;
     opt.gate_scale = gate_scale;
     opt.eps = norm_eps;
-    return launch_lean(a, g_workspace, g_workspace_bytes, reinterpret_cast<cudaStream_t>(stream), opt);
+    return launch_lean(a, ws.ptr, ws.bytes, reinterpret_cast<cudaStream_t>(stream), opt);
 }
 
 size_t gdn_workspace_bytes(int B, int T, int H, int d_k, int d_v, int packed) {
@@ -299,13 +315,17 @@ size_t gdn_workspace_bytes(int B, int T, int H, int d_k, int d_v, int packed) {
 
 int gdn_set_workspace(void* device_ptr, size_t bytes) {
     if (device_ptr && (reinterpret_cast<uintptr_t>(device_ptr) & 255u)) return GDN_ERR_UNSUPPORTED;
-    g_workspace = nullptr;
-    g_workspace_bytes = 0;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return device_ptr ? GDN_ERR_CUDA : GDN_OK;   // no device: nothing was set
+    if (dev < 0 || dev >= kMaxDevices) return GDN_ERR_UNSUPPORTED;
+    Workspace ws;
     if (device_ptr && bytes >= 4096) {
         if (int rc = lean_init_workspace(device_ptr)) return rc;
-        g_workspace = device_ptr;
-        g_workspace_bytes = bytes;
+        ws.ptr = device_ptr;
+        ws.bytes = bytes;
     }
+    std::lock_guard<std::mutex> lock(g_workspace_mutex);
+    g_workspace_of_device[dev] = ws;
     return GDN_OK;
 }
 
@@ -323,6 +343,17 @@ int gdn_query_status(void) {
     return s ? s : attn_query_status();
 }
 
+int gdn_query_status_stream(gdn_stream_t stream_) {
+    cudaStream_t stream = reinterpret_cast<cudaStream_t>(stream_);
+    int words[3] = {0, 0, 0};
+    if (tc_status_async(&words[0], stream) || lean_status_async(&words[1], stream) || attn_status_async(&words[2], stream))
+        return GDN_ERR_CUDA;
+    if (cudaStreamSynchronize(stream) != cudaSuccess) return GDN_ERR_CUDA;
+    for (int w : words)
+        if (w) return w;
+    return GDN_OK;
+}
+
 // Not part of the public header: 0 = automatic, 1 = fused kernel only, 2 = two-kernel pipeline only.
 void gdn_debug_force_path(int path) { g_force_path = path; }
 
@@ -337,9 +368,10 @@ int gdn_debug_set_timing(int enable) { return lean_set_timing(enable); }
 int gdn_debug_get_timing(float* ms5) { return ms5 ? lean_get_timing(ms5) : GDN_ERR_INVALID_ARG; }
 
 // Not part of the public header: forces the number of sequence segments (0 = automatic); chooses between the
-// merged scan kernel (1, default: used whenever its grid fits the GPU at once) and the three stand-alone kernels (0).
+// merged scan kernel (1: used whenever its grid fits the GPU at once) and the three stand-alone kernels (0, default).
 void gdn_debug_force_segments(int nseg) { lean_force_segments(nseg); }
 void gdn_debug_set_scan(int enable) { lean_set_scan(enable); }
+void gdn_debug_set_l2_hints(int enable) { lean_set_l2_hints(enable); }
 
 // Not part of the public header: lets the tests capture per-stage intermediates.
 void gdn_debug_set_dump(float* device_buffer) { tc_set_debug_dump(device_buffer); }

@@ -1,4 +1,4 @@
-// Single-token decode step of the gated delta rule (the recurrence "updated token-by-token",
+// Single-token decode step of the gated delta rule (the recurrence advanced by one token,
 // Section "The model"; decode is bandwidth-bound, Section "Decode, and why 4-bit is slower").
 //
 // Per (sequence, head), state S in R^{d_k x d_v} (fp32, updated in place), one token:

@@ -34,6 +34,11 @@ bool simt_supported(int d_k, int d_v);
 int launch_tc(const PrefillArgs& a, cudaStream_t stream);
 bool tc_supported(int d_k, int d_v);
 int tc_query_status();               // synchronises the device, returns the kernels' status word
+// Enqueue, on `stream`, the copy of one translation unit's status word to *host_dst (read it after the stream
+// has been synchronised).
+int tc_status_async(int* host_dst, cudaStream_t stream);
+int lean_status_async(int* host_dst, cudaStream_t stream);
+int attn_status_async(int* host_dst, cudaStream_t stream);
 void tc_set_debug_dump(float* p);    // tests only: stage dump of chunk 0 of CTA (0,0,0)
 
 // [tokens, H, d] bf16 tensor map, box = 64 tokens x 1 head x 64 features, 128-byte swizzle
@@ -59,6 +64,7 @@ int lean_reset_status();              // tests only: clear the status word
 void lean_set_debug(float* p);        // tests only: time stamps of the chain kernel
 int lean_set_timing(int enable);      // benchmark only: record events around each kernel
 int lean_get_timing(float* ms5);      // {prepare, summary, combine, chain, scan} of the last call
+void lean_set_l2_hints(int enable);   // tests only: 0 = no L2 eviction-priority hints
 void lean_set_scan(int enable);       // tests only: 0 = never merge summary, combine and chain into one launch
 
 // Single-token decode step (bf16 q/k/v/out, fp32 state updated in place).

@@ -41,7 +41,10 @@ static cudaEvent_t g_lean_events[5] = {nullptr, nullptr, nullptr, nullptr, nullp
 static bool g_lean_split_last = false;
 static float* g_lean_dbg = nullptr;        // debug: time stamps of the chain kernel
 static int g_lean_drop_chunk = -1;         // tests: chunk the chain kernel's TMA thread skips (-1 = none)
-static bool g_lean_use_scan = true;        // tests: false = always the stand-alone summary / combine / chain kernels
+static int g_lean_l2_hints = 1;            // tests: 0 = no L2 eviction-priority hints on the tile loads
+static bool g_lean_use_scan = false;       // true = summary, combination and chain of a split run as one resident launch (measured
+                                           // slower than the three kernels under programmatic dependent launch: 0.162 vs 0.152 ms on
+                                           // the 10240-token workload, 0.074 vs 0.060 ms at 2048 tokens, so it is off by default)
 static bool g_lean_scan_last = false;
 
 namespace {
@@ -172,6 +175,7 @@ struct PrepParams {
     int B, T, H;
     float gate_scale, eps;     // raw inputs only
     int* ticket;               // {next item, CTAs done}: both zero before the launch, both zero again after it
+    int l2;                    // 1: the K tiles are read again by later kernels of this call and fit in L2: keep them there
 };
 
 constexpr uint32_t ID_G = make_idesc(128, 64, kFmtBF16, kFmtBF16, kMajorK, kMajorK);
@@ -200,7 +204,7 @@ __device__ __forceinline__ bool decode_item(const PrepParams& p, long item, int*
 }
 
 // RAW: q and k are raw projections and a, beta pre-activations.  The norms and the gating
-// (Section "Batched prefill": per-position kernels around the projections) are folded in here: the
+// (Section "Prefill projections: dequantize, then call the vendor": per-position kernels around the projections) are folded in here: the
 // inverse row norms scale A, P and the columns of T diag(b e^g), and they ride to the chain kernels
 // inside the gate vectors (e^g / |q| for the output rows, e^{gC-g} / |k| for the state update), so
 // the K and Q tiles themselves are used as they are.
@@ -538,11 +542,17 @@ gdn_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             // ================= TMA + MMA issue (one thread) =================
             if (lane == 0) {
                 const uint32_t kq = base + PS_KQ, full = w.bar(PB_FULL);
+                const uint64_t pol_keep = l2_policy_evict_last();
                 auto load_tiles = [&](int hh, long tk) {
                     mbar_arrive_expect_tx(full, 32768);
-                    tma_load_3d(kq, &map_k, 0, hh, (int)tk, full);
+                    if (p.l2) {
+                        tma_load_3d_hint(kq, &map_k, 0, hh, (int)tk, full, pol_keep);
+                        tma_load_3d_hint(kq + 16384, &map_k, 64, hh, (int)tk, full, pol_keep);
+                    } else {
+                        tma_load_3d(kq, &map_k, 0, hh, (int)tk, full);
+                        tma_load_3d(kq + 16384, &map_k, 64, hh, (int)tk, full);
+                    }
                     tma_load_3d(kq + 8192, &map_q, 0, hh, (int)tk, full);
-                    tma_load_3d(kq + 16384, &map_k, 64, hh, (int)tk, full);
                     tma_load_3d(kq + 24576, &map_q, 64, hh, (int)tk, full);
                 };
                 if (it == 0) load_tiles(h, tok);                    // later items were requested one item ahead
@@ -659,6 +669,7 @@ struct ChainParams {
     int nseg, seg_chunks;     // segments per sequence (1 = no split) and chunks per segment
     float* snaps;             // optional [B, nsnap, H, d_k, d_v]: the state after every snap_every chunks
     int snap_every, nsnap;
+    int l2;                   // 1: the K, Q, V tiles are read for the last time here: mark them first to be evicted
 };
 
 // One CTA's identity inside a kernel: aligned shared-memory base (address and pointer), tensor-memory base,
@@ -961,6 +972,7 @@ __device__ __forceinline__ void chain_body(const CUtensorMap* map_q, const CUten
             prefetch_tensormap(map_q);
             prefetch_tensormap(map_k);
             prefetch_tensormap(map_v);
+            const uint64_t pol_done = l2_policy_evict_first();
             for (int c = 0; c < nchunks; ++c) {
                 if (c == p.drop_chunk && dvb == 0 && h == 0 && cta.z == 0) continue;
                 const int tok = (int)(tok0 + (long)c * C);
@@ -969,8 +981,13 @@ __device__ __forceinline__ void chain_body(const CUtensorMap* map_q, const CUten
                     const uint32_t sB = c % 3, bb = base + CS_B + sB * STAGE_B, full = w.bar(CB_FULLB0 + sB);
                     if (c >= 3) w.wait(CB_FREEB0 + sB, ((c / 3) - 1) & 1);
                     mbar_arrive_expect_tx(full, STAGE_B_TX);
-                    tma_load_3d(bb + ST_V, map_v, dvb * DVB, h, tok, full);
-                    tma_load_3d(bb + ST_V + 8192, map_v, dvb * DVB + 64, h, tok, full);
+                    if (p.l2) {
+                        tma_load_3d_hint(bb + ST_V, map_v, dvb * DVB, h, tok, full, pol_done);
+                        tma_load_3d_hint(bb + ST_V + 8192, map_v, dvb * DVB + 64, h, tok, full, pol_done);
+                    } else {
+                        tma_load_3d(bb + ST_V, map_v, dvb * DVB, h, tok, full);
+                        tma_load_3d(bb + ST_V + 8192, map_v, dvb * DVB + 64, h, tok, full);
+                    }
                     bulk_load(bb + ST_T2, item + IT_T2, 8192, full);
                 }
                 {   // ring A: K/Q tiles, -W^T, P, and the gate vectors (own 4-deep ring, same barrier)
@@ -978,10 +995,17 @@ __device__ __forceinline__ void chain_body(const CUtensorMap* map_q, const CUten
                     if (c >= 2) w.wait(CB_FREEA0 + s, ((c >> 1) - 1) & 1);
                     mbar_arrive_expect_tx(full, STAGE_A_TX);
                     bulk_load(sb + ST_W, item + IT_W, 16384, full);
-                    tma_load_3d(sb + ST_KQ, map_k, 0, h, tok, full);
-                    tma_load_3d(sb + ST_KQ + 8192, map_q, 0, h, tok, full);
-                    tma_load_3d(sb + ST_KQ + 16384, map_k, 64, h, tok, full);
-                    tma_load_3d(sb + ST_KQ + 24576, map_q, 64, h, tok, full);
+                    if (p.l2) {
+                        tma_load_3d_hint(sb + ST_KQ, map_k, 0, h, tok, full, pol_done);
+                        tma_load_3d_hint(sb + ST_KQ + 8192, map_q, 0, h, tok, full, pol_done);
+                        tma_load_3d_hint(sb + ST_KQ + 16384, map_k, 64, h, tok, full, pol_done);
+                        tma_load_3d_hint(sb + ST_KQ + 24576, map_q, 64, h, tok, full, pol_done);
+                    } else {
+                        tma_load_3d(sb + ST_KQ, map_k, 0, h, tok, full);
+                        tma_load_3d(sb + ST_KQ + 8192, map_q, 0, h, tok, full);
+                        tma_load_3d(sb + ST_KQ + 16384, map_k, 64, h, tok, full);
+                        tma_load_3d(sb + ST_KQ + 24576, map_q, 64, h, tok, full);
+                    }
                     bulk_load(sb + ST_P, item + IT_P, 8192, full);
                     bulk_load(base + CS_GATES + (c & 3) * 1280, item + IT_GATES, 1280, full);
                 }
@@ -1072,6 +1096,7 @@ struct SummaryParams {
     float* seg_mt;            // [B*nseg, H] x 64 KiB: M_seg^T as two bf16 operand images (leading part | remainder)
     int B, T, H, dv;
     int nseg, seg_chunks;
+    int l2;                   // 1: K and V are read again by the chain phase and fit in L2: keep them there
 };
 
 __device__ __forceinline__ void summary_init_bars(const Waiter& w, int ninst) {
@@ -1235,6 +1260,7 @@ __device__ __forceinline__ void summary_body(const CUtensorMap* map_k, const CUt
         } else if (warp == 9 && lane == 0) {
             prefetch_tensormap(map_k);
             prefetch_tensormap(map_v);
+            const uint64_t pol_keep = l2_policy_evict_last();
             for (int c = 0; c < nchunks; ++c) {
                 const uint32_t s = c % SUM_STAGES, sb = base + s * SUM_STAGE;
                 if (c >= (int)SUM_STAGES) w.wait(SB_FREE0 + s, ((c / SUM_STAGES) - 1) & 1);
@@ -1242,10 +1268,17 @@ __device__ __forceinline__ void summary_body(const CUtensorMap* map_k, const CUt
                 const int tok = (int)(tok0 + (long)c * C);
                 const uint8_t* item = p.items + (size_t)((slot0 + c) * H + h) * ITEM_BYTES;
                 mbar_arrive_expect_tx(full, SUM_STAGE_TX);
-                tma_load_3d(sb + SS_K, map_k, 0, h, tok, full);
-                tma_load_3d(sb + SS_K + 8192, map_k, 64, h, tok, full);
-                tma_load_3d(sb + SS_V, map_v, dvb * DVB, h, tok, full);
-                tma_load_3d(sb + SS_V + 8192, map_v, dvb * DVB + 64, h, tok, full);
+                if (p.l2) {
+                    tma_load_3d_hint(sb + SS_K, map_k, 0, h, tok, full, pol_keep);
+                    tma_load_3d_hint(sb + SS_K + 8192, map_k, 64, h, tok, full, pol_keep);
+                    tma_load_3d_hint(sb + SS_V, map_v, dvb * DVB, h, tok, full, pol_keep);
+                    tma_load_3d_hint(sb + SS_V + 8192, map_v, dvb * DVB + 64, h, tok, full, pol_keep);
+                } else {
+                    tma_load_3d(sb + SS_K, map_k, 0, h, tok, full);
+                    tma_load_3d(sb + SS_K + 8192, map_k, 64, h, tok, full);
+                    tma_load_3d(sb + SS_V, map_v, dvb * DVB, h, tok, full);
+                    tma_load_3d(sb + SS_V + 8192, map_v, dvb * DVB + 64, h, tok, full);
+                }
                 bulk_load(sb + SS_W, item + IT_W, 16384, full);
                 bulk_load(sb + SS_T2, item + IT_T2, 8192, full);
                 bulk_load(sb + SS_GATES, item + IT_GATES, 1280, full);
@@ -1561,7 +1594,9 @@ gdn_scan_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             tc_fence_before_sync();
             cta_sync();
             tc_fence_after_sync();
-            if (tid == 0) { __threadfence(); atomicAdd(fl + 0, 1); }
+            // (test hook: drop_chunk == -2 makes the first CTA keep its summary to itself, so that the
+            //  bounded waits of its head on this counter expire)
+            if (tid == 0 && !(p.cp.drop_chunk == -2 && blockIdx.y == 0 && blockIdx.z == 0)) { __threadfence(); atomicAdd(fl + 0, 1); }
         }
         stamp(1);
         // ---------------- phase 2: the hops of this CTA's column slices ----------------
@@ -1754,7 +1789,10 @@ int launch_lean(const PrefillArgs& a, void* workspace, size_t workspace_bytes, c
     const long nslots = (long)(tokens >> 6) + a.B;
     const long nitems = nslots * a.H;
     // ---- state-independent steps, every (chunk, head) ----
-    PrepParams pp{a.log_alpha, a.beta, a.cu_seqlens, ws, nslots, a.B, a.T, a.H, opt.gate_scale, opt.eps, ticket};
+    // With a split, K (and V) are read by two or three kernels of the call; when they fit in L2 comfortably the
+    // earlier readers ask L2 to keep them and the last reader releases them.
+    const int l2 = (g_lean_l2_hints && nseg > 1 && tokens * a.H * (uint64_t)(a.d_k + a.d_v) * 2 <= (96ull << 20)) ? 1 : 0;
+    PrepParams pp{a.log_alpha, a.beta, a.cu_seqlens, ws, nslots, a.B, a.T, a.H, opt.gate_scale, opt.eps, ticket, l2};
     const int pgrid = (int)(nitems < 4L * num_sms ? nitems : 4L * num_sms);
     auto mark = [&](int i) { if (g_lean_timing && g_lean_events[i]) cudaEventRecord(g_lean_events[i], stream); };
     mark(0);
@@ -1773,13 +1811,13 @@ int launch_lean(const PrefillArgs& a, void* workspace, size_t workspace_bytes, c
         seg_sin = reinterpret_cast<float*>(ws + items_bytes);
         float* seg_n = seg_sin + state_elems;
         float* seg_mt = seg_n + state_elems;
-        SummaryParams sp{a.cu_seqlens, ws, seg_n, seg_mt, a.B, a.T, a.H, a.d_v, nseg, seg_chunks};
+        SummaryParams sp{a.cu_seqlens, ws, seg_n, seg_mt, a.B, a.T, a.H, a.d_v, nseg, seg_chunks, l2};
         CombineParams cb{a.initial_state, seg_n, seg_mt, seg_sin, a.H, a.d_v, nseg};
         // one resident CTA per (sequence, head, segment) runs all three phases when the grid fits the GPU at once
         if (g_lean_use_scan && a.d_v == DVB && (long)a.B * a.H * nseg <= num_sms && (long)a.B * a.H <= kMaxScanChains) {
             ChainParams cp{a.initial_state, static_cast<__nv_bfloat16*>(a.out), a.final_state, a.cu_seqlens,
                            ws, seg_sin, g_lean_dbg, g_lean_drop_chunk, a.B, a.T, a.H, a.d_v, nseg, seg_chunks,
-                           snaps, snap_every, nsnap};
+                           snaps, snap_every, nsnap, l2};
             ScanParams scp{sp, cb, cp, static_cast<int*>(workspace) + kScanFlagOffset};
             dim3 grid(1, a.H, a.B * nseg);
             if (g_lean_dbg) launch_after(gdn_scan_kernel<true>, grid, SCAN_THREADS, SCAN_SMEM, stream, mq, mk, mv, scp);
@@ -1803,7 +1841,7 @@ int launch_lean(const PrefillArgs& a, void* workspace, size_t workspace_bytes, c
     // ---- steps c, d ----
     ChainParams cp{a.initial_state, static_cast<__nv_bfloat16*>(a.out), a.final_state, a.cu_seqlens,
                    ws, seg_sin, g_lean_dbg, g_lean_drop_chunk, a.B, a.T, a.H, a.d_v, nseg, seg_chunks,
-                   snaps, snap_every, nsnap};
+                   snaps, snap_every, nsnap, l2};
     dim3 grid(a.d_v / DVB, a.H, a.B * nseg);
     if (g_lean_dbg) launch_after(gdn_chain_kernel<true>, grid, CHAIN_THREADS, CHAIN_SMEM, stream, mq, mk, mv, cp);
     else launch_after(gdn_chain_kernel<false>, grid, CHAIN_THREADS, CHAIN_SMEM, stream, mq, mk, mv, cp);
@@ -1813,6 +1851,7 @@ int launch_lean(const PrefillArgs& a, void* workspace, size_t workspace_bytes, c
 }
 
 void lean_set_scan(int enable) { g_lean_use_scan = enable != 0; }
+void lean_set_l2_hints(int enable) { g_lean_l2_hints = enable; }
 void lean_force_segments(int nseg) { g_lean_force_nseg = nseg; }
 void lean_set_debug(float* p) { g_lean_dbg = p; }
 void lean_set_drop_chunk(int c) { g_lean_drop_chunk = c; }
@@ -1917,6 +1956,11 @@ int launch_lean_static(const PrefillArgs& a, cudaStream_t stream) {
     gdn_chain_kernel<false><<<grid, CHAIN_THREADS, CHAIN_SMEM, stream>>>(mq, mk, mv, cp);
     count_launch();
     return cudaGetLastError() == cudaSuccess ? GDN_OK : GDN_ERR_CUDA;
+}
+
+int lean_status_async(int* host_dst, cudaStream_t stream) {
+    return cudaMemcpyFromSymbolAsync(host_dst, g_lean_status, sizeof(int), 0, cudaMemcpyDeviceToHost, stream) == cudaSuccess
+               ? GDN_OK : GDN_ERR_CUDA;
 }
 
 int lean_query_status() {

@@ -803,6 +803,11 @@ int tc_query_status() {
     return s ? s : lean_query_status();
 }
 
+int tc_status_async(int* host_dst, cudaStream_t stream) {
+    return cudaMemcpyFromSymbolAsync(host_dst, g_tc_status, sizeof(int), 0, cudaMemcpyDeviceToHost, stream) == cudaSuccess
+               ? GDN_OK : GDN_ERR_CUDA;
+}
+
 void tc_set_debug_dump(float* p) { g_debug_dump = p; }
 
 }  // namespace gdn

@@ -10,14 +10,16 @@ from gdn_testlib import to_device
 pytestmark = pytest.mark.gpu
 
 
-@pytest.mark.parametrize("T,nseg", [(64 * 6 + 11, 0), (64 * 20, 4)])      # plain two-kernel path, sequence split
-def test_captured_call_replays(T, nseg):
+# plain two-kernel path, sequence split as three kernels, sequence split as one merged launch
+@pytest.mark.parametrize("T,nseg,merged", [(64 * 6 + 11, 0, 0), (64 * 20, 4, 0), (64 * 20, 4, 1)])
+def test_captured_call_replays(T, nseg, merged):
     import paper_2607_14568_b200 as gdn
     cfg = get_config("short", B=1, T=T, H=2, init_std=0.2)
     d = to_device(make_inputs(cfg))
     ws = torch.empty(gdn.gdn_workspace_bytes(1, T, 2, cfg.d_k, cfg.d_v, False), dtype=torch.uint8, device="cuda")
     gdn.gdn_set_workspace(ws)
     gdn.lib().gdn_debug_force_segments(nseg)
+    gdn.lib().gdn_debug_set_scan(merged)
     try:
         def call():
             gdn.gdn_chunk_prefill(d["q"], d["k"], d["v"], d["log_alpha"], d["beta"], d["initial_state"], d["out"],
@@ -50,4 +52,5 @@ def test_captured_call_replays(T, nseg):
         assert not torch.equal(got_out, want_out)
     finally:
         gdn.lib().gdn_debug_force_segments(0)
+        gdn.lib().gdn_debug_set_scan(0)
         gdn.gdn_set_workspace(None)

@@ -131,7 +131,7 @@ def test_two_kernel_sequence_split(T, nseg, gate, merged):
         check_bf16(x, prefill_two_kernel, f"split T={T} nseg={nseg} merged={merged}, second call")   # counters were left clean
     finally:
         gdn.lib().gdn_debug_force_segments(0)
-        gdn.lib().gdn_debug_set_scan(1)
+        gdn.lib().gdn_debug_set_scan(0)
 
 
 def test_two_kernel_sequence_split_wide_values_and_batch():
@@ -215,9 +215,9 @@ def test_bf16_large_all_chains(impl):
 
 
 # ---- final_state written over initial_state ------------------------------------------------------------
-@pytest.mark.parametrize("impl,nseg,H", [("fused", 0, 4), ("two_kernel", 0, 4), ("two_kernel", 3, 64),
-                                         ("two_kernel", 16, 16), ("two_kernel", 9, 16)])
-def test_bf16_final_state_may_alias_initial_state(impl, nseg, H):
+@pytest.mark.parametrize("impl,nseg,H,merged", [("fused", 0, 4, 0), ("two_kernel", 0, 4, 0), ("two_kernel", 3, 64, 0),
+                                                ("two_kernel", 16, 16, 0), ("two_kernel", 9, 16, 1)])
+def test_bf16_final_state_may_alias_initial_state(impl, nseg, H, merged):
     """The header allows final_state == initial_state.  With the sequence split the grid of the last kernel
     (H * nseg CTAs: 192 and 256 in two of the cases) does not fit the GPU in one wave, so a segment-0 CTA may well
     start after a last-segment CTA has finished; 16 heads x 9 segments run as the merged single launch.  The result
@@ -227,10 +227,12 @@ def test_bf16_final_state_may_alias_initial_state(impl, nseg, H):
     d = to_device(x)
     d["final_state"] = d["initial_state"]
     gdn.lib().gdn_debug_force_segments(nseg)
+    gdn.lib().gdn_debug_set_scan(merged)
     try:
         out, fin = run_lib(BF16_FNS[impl], d)
     finally:
         gdn.lib().gdn_debug_force_segments(0)
+        gdn.lib().gdn_debug_set_scan(0)
     o_ref, f_ref = run_oracle(x)
     assert_close(f64(out), o_ref, BF16_REL_L2, BF16_MAX_ABS, "aliased out")
     assert_close(f64(fin), f_ref, BF16_REL_L2, BF16_MAX_ABS, "aliased final_state")

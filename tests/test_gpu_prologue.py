@@ -1,5 +1,5 @@
-"""Prefill on raw projections (norms and gating fused into the prepare kernel; Section "Batched
-prefill") against the fp64 oracle: oracle.prologue followed by the token-by-token recurrence."""
+"""Prefill on raw projections (norms and gating fused into the prepare kernel; Section "Prefill
+projections: dequantize, then call the vendor") against the fp64 oracle: oracle.prologue followed by the token-by-token recurrence."""
 import numpy as np
 import pytest
 import torch

@@ -266,3 +266,61 @@ def test_prologue_invariants():
     from scipy.special import expit, log1p, logsumexp  # noqa: F401
     np.testing.assert_allclose(be, expit(b_raw), rtol=1e-14)
     np.testing.assert_allclose(la, -0.05 * np.logaddexp(0.0, a_raw), rtol=1e-13)
+
+
+# --- stage outputs of the chunked form: each against something that is not the chunked code ------------
+def test_chunked_stages_against_token_loop_and_linear_algebra():
+    """oracle.chunked_stages hands out g, A, P, T, W, U, Delta and the incoming state of every chunk of one
+    chain.  Delta and the states are pinned by a token-by-token loop written here (the per-token correction
+    delta_t and the state at each chunk boundary are what the recurrence itself produces); T by (I + A) T = I;
+    g, A, P, W, U by numpy expressions of their definitions on the raw inputs; the outputs and the final state
+    by the sequential oracle.  A packed batch with a ragged tail, chain (1, 1)."""
+    rng = np.random.default_rng(11)
+    H, dk, dv, C = 2, 8, 6, 16
+    lengths = [20, 37, 5]
+    cu = np.concatenate([[0], np.cumsum(lengths)]).astype(np.int32)
+    Tt = int(cu[-1])
+    q, k, v, la, beta, S0 = rand_problem(rng, B=1, T=Tt, H=H, dk=dk, dv=dv)
+    q, k, v, la, beta = q[0], k[0], v[0], la[0], beta[0]                 # packed [T,H,.]
+    S0 = rng.standard_normal((3, H, dk, dv)) * 0.5
+    n, h = 1, 1
+    st = oracle.chunked_stages(q, k, v, la, beta, S0, cu, chunk=C, n=n, h=h)
+    L = lengths[n]
+    a, b = int(cu[n]), int(cu[n + 1])
+    kk, qq, vv, aa, bb = k[a:b, h], q[a:b, h], v[a:b, h], la[a:b, h], beta[a:b, h]
+    # token loop: deltas, boundary states, outputs
+    S = S0[n, h].copy()
+    deltas, outs, bounds = [], [], []
+    for t in range(L):
+        if t % C == 0:
+            bounds.append(S.copy())
+        S = np.exp(aa[t]) * S
+        d = bb[t] * (vv[t] - S.T @ kk[t])
+        S = S + np.outer(kk[t], d)
+        deltas.append(d)
+        outs.append(S.T @ qq[t])
+    nch = (L + C - 1) // C
+    assert st["length"] == L and st["g"].shape == (nch, C)
+    assert rel(st["out"], np.array(outs)) < RTOL and rel(st["final_state"], S) < RTOL
+    seq_out, seq_fin = oracle.sequential(q, k, v, la, beta, S0, cu)
+    assert rel(st["out"], seq_out[a:b, h]) < RTOL and rel(st["final_state"], seq_fin[n, h]) < RTOL
+    for c in range(nch):
+        R = min(C, L - c * C)
+        sl = slice(c * C, c * C + R)
+        g = np.cumsum(aa[sl])
+        assert rel(st["g"][c, :R], g) < RTOL
+        assert rel(st["S_in"][c], bounds[c]) < RTOL
+        assert rel(st["Delta"][c, :R], np.array(deltas[c * C:c * C + R])) < 1e-11
+        dec = np.exp(g[:, None] - g[None, :])
+        A = np.tril(bb[sl, None] * dec * (kk[sl] @ kk[sl].T), -1)
+        P = np.tril(dec * (qq[sl] @ kk[sl].T), 0)
+        assert rel(st["A"][c, :R, :R], A) < RTOL and rel(st["P"][c, :R, :R], P) < RTOL
+        T = st["T"][c, :R, :R]
+        assert np.abs((np.eye(R) + A) @ T - np.eye(R)).max() < 1e-12
+        assert np.abs(np.triu(T, 1)).max() == 0.0 and np.allclose(np.diag(T), 1.0)
+        assert rel(st["W"][c, :R], T @ (bb[sl, None] * np.exp(g)[:, None] * kk[sl])) < RTOL
+        assert rel(st["U"][c, :R], T @ (bb[sl, None] * vv[sl])) < RTOL
+        # the chunk's correction is U - W S_in (what the GPU chain forms)
+        assert rel(st["Delta"][c, :R], st["U"][c, :R] - st["W"][c, :R] @ st["S_in"][c]) < 1e-11
+        # rows beyond a ragged tail stay zero
+        assert not st["W"][c, R:].any() and not st["T"][c, R:].any()
