@@ -3,5 +3,5 @@
 Nothing in the product package may import this; only the tests, the smoke check
 and the CPU-baseline leg of the benchmark do.
 """
-from .gdn_oracle import (chunked, chunked_stages, dense, num_threads, prologue, sequential)  # noqa: F401
+from .gdn_oracle import (chunked, chunked_stages, dense, epilogue, num_threads, prologue, sequential)  # noqa: F401
 from .attn_oracle import attention_causal, attention_causal_rows, attention_gemm_form  # noqa: F401

@@ -19,6 +19,10 @@ the C file: ``q,k [B,T,H,d_k]``, ``v [B,T,H,d_v]``, ``log_alpha,beta [B,T,H]``,
               axis, beta = sigmoid(b), log_alpha = -softplus(a) * gate_scale.  The paper names
               these kernels without printing formulas; the forms here are the reading the
               benchmark inputs were drawn with.  Plain numpy, fp64.
+  epilogue    the per-position kernels behind the scan (same section: "norms ... gating" are batched
+              over the chunk): a root-mean-square norm of each output row over the value axis with a
+              learned weight vector, multiplied by the SiLU of a gate tensor.  Again the paper prints no
+              formula; this is the reading recorded for the fused output stage.  Plain numpy, fp64.
 """
 from __future__ import annotations
 
@@ -146,3 +150,13 @@ def prologue(q_raw, k_raw, a_raw, b_raw, gate_scale, eps=0.0):
     beta = 1.0 / (1.0 + np.exp(-b_raw))
     log_alpha = -np.log(1.0 + np.exp(a_raw)) * float(gate_scale)
     return q, k, log_alpha, beta
+
+
+def epilogue(o, z, weight, eps=0.0):
+    """Gated output norm per (token, head) over the value axis (last axis, length d_v):
+    o / sqrt(mean_j o_j^2 + eps) * weight * silu(z),  silu(z) = z / (1 + e^{-z});  weight has shape [d_v]."""
+    o, z, weight = _f64(o), _f64(z), _f64(weight)
+    if z.shape != o.shape or weight.shape != (o.shape[-1],):
+        raise ValueError("z must have the shape of o and weight the length of its last axis")
+    rms = np.sqrt((o * o).mean(axis=-1, keepdims=True) + float(eps))
+    return o / rms * weight * (z / (1.0 + np.exp(-z)))

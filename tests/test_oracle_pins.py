@@ -324,3 +324,50 @@ def test_chunked_stages_against_token_loop_and_linear_algebra():
         assert rel(st["Delta"][c, :R], st["U"][c, :R] - st["W"][c, :R] @ st["S_in"][c]) < 1e-11
         # rows beyond a ragged tail stay zero
         assert not st["W"][c, R:].any() and not st["T"][c, R:].any()
+
+
+# --- epilogue (gated root-mean-square norm behind the scan) --------------------------------------------
+def test_epilogue_closed_forms():
+    import math
+    # rows (3, 4) and (6, 8, 0, 0): mean squares 12.5 and 25; gates 0, ln 3 (silu = ln 3 * 3/4) and large
+    o = np.array([[3.0, 4.0]])
+    out = oracle.epilogue(o, np.array([[math.log(3.0), 0.0]]), np.array([1.0, 1.0]))
+    np.testing.assert_allclose(out, [[3.0 / math.sqrt(12.5) * math.log(3.0) * 0.75, 0.0]], rtol=1e-14)
+    o = np.array([[6.0, 8.0, 0.0, 0.0]])
+    z = np.array([[40.0, -40.0, 1.0, 2.0]])                # silu(40) = 40 to 1e-16, silu(-40) = -40 e^-40
+    out = oracle.epilogue(o, z, np.array([2.0, 3.0, 5.0, 7.0]))
+    np.testing.assert_allclose(out[0, 0], 6.0 / 5.0 * 2.0 * 40.0, rtol=1e-14)
+    np.testing.assert_allclose(out[0, 1], 8.0 / 5.0 * 3.0 * (-40.0 * math.exp(-40.0) / (1 + math.exp(-40.0))), rtol=1e-12)
+    assert out[0, 2] == 0.0 and out[0, 3] == 0.0
+    # eps under the root: mean square 25 + eps 11 = 36
+    out = oracle.epilogue(o, np.full((1, 4), 40.0), np.ones(4), eps=11.0)
+    np.testing.assert_allclose(out[0, :2], [40.0, 8.0 / 6.0 * 40.0], rtol=1e-14)
+
+
+def test_epilogue_invariants_and_scalar_loops():
+    import math
+    rng = np.random.default_rng(21)
+    o = rng.standard_normal((2, 5, 3, 8))
+    z = rng.standard_normal((2, 5, 3, 8))
+    w = rng.standard_normal(8)
+    out = oracle.epilogue(o, z, w, eps=1e-3)
+    assert out.shape == o.shape
+    # scalar loops that know nothing of numpy broadcasting
+    for idx in [(0, 0, 0), (1, 4, 2), (0, 3, 1)]:
+        row, gate = o[idx], z[idx]
+        ms = sum(x * x for x in row) / 8 + 1e-3
+        for j in range(8):
+            want = row[j] / math.sqrt(ms) * w[j] * gate[j] / (1.0 + math.exp(-gate[j]))
+            assert abs(out[idx][j] - want) <= 1e-13 * max(1.0, abs(want))
+    # the norm removes the scale of o (eps = 0), every row has unit mean square before weight and gate
+    a = oracle.epilogue(o, z, w)
+    b = oracle.epilogue(o * 7.5, z, w)
+    assert rel(a, b) < RTOL
+    unit = oracle.epilogue(o, np.full(o.shape, 60.0), np.ones(8)) / 60.0
+    np.testing.assert_allclose((unit * unit).mean(axis=-1), 1.0, rtol=1e-12)
+    # linear in the weight; rows and heads are independent
+    assert rel(oracle.epilogue(o, z, 2.0 * w), 2.0 * a) < RTOL
+    assert rel(oracle.epilogue(o[:, 2:3, 1:2], z[:, 2:3, 1:2], w), a[:, 2:3, 1:2]) < RTOL
+    # silu(z) + silu(-z) = z (2 sigma(z) - 1) ... pinned through silu(z) - silu(-z) = z
+    c = oracle.epilogue(o, -z, w)
+    assert rel(a - c, oracle.epilogue(o, np.full(o.shape, 60.0), w) / 60.0 * z) < 1e-12
