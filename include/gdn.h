@@ -191,6 +191,27 @@ int gdn_chunk_prefill_raw(const void* q_raw, const void* k_raw, const void* v,
                           gdn_stream_t stream);
 
 /*
+ * gdn_chunk_prefill with the per-position output stage fused in (Section "Prefill projections:
+ * dequantize, then call the vendor" names the norms and the gating that surround the scan among the
+ * kernels batched over the chunk; the paper prints no formula, this library takes the gated
+ * root-mean-square norm).  Per (token, head), with o the row gdn_chunk_prefill would return,
+ *   out_j = o_j / sqrt(mean_j' o_j'^2 + norm_eps) * norm_weight_j * silu(gate_z_j),  silu(z) = z / (1 + e^{-z})
+ * gate_z is bf16 with the shape of out, norm_weight is fp32 [d_v] (shared by all heads), norm_eps >= 0.
+ * The norm is taken on the fp32 rows before they are rounded, inside the kernel that produces them, so
+ * the un-normalised output is never written.  Supported: d_k = d_v = 128, chunk = 64.  Needs the scratch of
+ * gdn_set_workspace (GDN_ERR_WORKSPACE without it).  final_state is the same as without the output stage.
+ * Errors: as gdn_chunk_prefill; GDN_ERR_INVALID_ARG for a NULL gate_z or norm_weight or a negative norm_eps.
+ */
+int gdn_chunk_prefill_gated(const void* q, const void* k, const void* v,
+                            const float* log_alpha, const float* beta,
+                            const float* initial_state,
+                            const void* gate_z, const float* norm_weight, float norm_eps,
+                            void* out, float* final_state,
+                            const int32_t* cu_seqlens,
+                            int B, int T, int H, int d_k, int d_v, int chunk,
+                            gdn_stream_t stream);
+
+/*
  * Optional scratch memory.  Without it gdn_chunk_prefill runs one fused kernel per call in
  * which each (sequence, head) chain also does its own forward substitutions.  With scratch of
  * at least gdn_workspace_bytes(...) bytes the state-independent steps (cumulative gate,

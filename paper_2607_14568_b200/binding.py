@@ -52,6 +52,8 @@ def lib():
         L.gdn_chunk_prefill_snapshots.restype = i
         L.gdn_chunk_prefill_raw.argtypes = [vp] * 5 + [ctypes.c_float] * 2 + [vp] * 4 + [i] * 6 + [vp]
         L.gdn_chunk_prefill_raw.restype = i
+        L.gdn_chunk_prefill_gated.argtypes = [vp] * 8 + [ctypes.c_float] + [vp] * 3 + [i] * 6 + [vp]
+        L.gdn_chunk_prefill_gated.restype = i
         L.gdn_attn_causal_prefill.argtypes = [vp] * 5 + [i] * 5 + [ctypes.c_float, vp]
         L.gdn_attn_causal_prefill.restype = i
         L.gdn_workspace_bytes.argtypes = [i] * 6
@@ -261,6 +263,27 @@ def gdn_chunk_prefill_raw(q_raw, k_raw, v, a_raw, b_raw, gate_scale, norm_eps, i
                                      _ptr(cu_seqlens), B, T, H, d_k, d_v, int(chunk), _stream(stream))
     if rc != 0:
         raise GdnError(rc, "gdn_chunk_prefill_raw")
+    return out, final_state
+
+
+def gdn_chunk_prefill_gated(q, k, v, log_alpha, beta, initial_state, gate_z, norm_weight, norm_eps, out, final_state,
+                            cu_seqlens=None, chunk: int = 64, stream=None):
+    """gdn_chunk_prefill with the output stage fused in: out = o / sqrt(mean o^2 + norm_eps) * norm_weight * silu(gate_z)
+    per (token, head); gate_z bf16 like out, norm_weight fp32 [d_v].  Needs gdn_set_workspace.  See include/gdn.h."""
+    f32, bf = torch.float32, torch.bfloat16
+    _check([("q", q, bf), ("k", k, bf), ("v", v, bf), ("out", out, bf), ("gate_z", gate_z, bf), ("log_alpha", log_alpha, f32),
+            ("beta", beta, f32), ("initial_state", initial_state, f32), ("final_state", final_state, f32),
+            ("norm_weight", norm_weight, f32), ("cu_seqlens", cu_seqlens, torch.int32)], bf, "cuda")
+    B, T, H, d_k, d_v = _dims(q, v, cu_seqlens)
+    if k.shape != q.shape or v.shape[:-1] != q.shape[:-1] or out.shape != v.shape or gate_z.shape != out.shape:
+        raise ValueError("q, k, v, gate_z, out shapes disagree")
+    if log_alpha.shape != q.shape[:-1] or beta.shape != q.shape[:-1] or tuple(norm_weight.shape) != (d_v,):
+        raise ValueError("gate or weight shapes disagree with q, v")
+    rc = lib().gdn_chunk_prefill_gated(_ptr(q), _ptr(k), _ptr(v), _ptr(log_alpha), _ptr(beta), _ptr(initial_state),
+                                       _ptr(gate_z), _ptr(norm_weight), float(norm_eps), _ptr(out), _ptr(final_state),
+                                       _ptr(cu_seqlens), B, T, H, d_k, d_v, int(chunk), _stream(stream))
+    if rc != 0:
+        raise GdnError(rc, "gdn_chunk_prefill_gated")
     return out, final_state
 
 

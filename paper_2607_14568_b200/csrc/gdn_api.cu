@@ -309,6 +309,26 @@ int gdn_chunk_prefill_raw(const void* q_raw, const void* k_raw, const void* v, c
     return launch_lean(a, ws.ptr, ws.bytes, reinterpret_cast<cudaStream_t>(stream), opt);
 }
 
+int gdn_chunk_prefill_gated(const void* q, const void* k, const void* v, const float* log_alpha, const float* beta,
+                            const float* initial_state, const void* gate_z, const float* norm_weight, float norm_eps,
+                            void* out, float* final_state, const int32_t* cu_seqlens, int B, int T, int H, int d_k,
+                            int d_v, int chunk, gdn_stream_t stream) {
+    const PrefillArgs a = pack(q, k, v, log_alpha, beta, initial_state, out, final_state, cu_seqlens, B, T, H, d_k, d_v);
+    if (int rc = validate(a, chunk)) return rc;
+    if (!gate_z || !norm_weight || !(norm_eps >= 0.f)) return GDN_ERR_INVALID_ARG;
+    if (!aligned16(gate_z) || !aligned16(norm_weight) || d_k != 128 || d_v != 128) return GDN_ERR_UNSUPPORTED;
+    const long tokens = cu_seqlens ? (long)T : (long)B * T;
+    if (tokens == 0) return launch_tc(a, reinterpret_cast<cudaStream_t>(stream));   // only copies the states
+    const size_t need = lean_workspace_bytes(B, T, H, d_k, d_v, cu_seqlens != nullptr);
+    const Workspace ws = current_workspace();
+    if (!ws.ptr || ws.bytes < need) return GDN_ERR_WORKSPACE;
+    LeanOptions opt;
+    opt.gate_z = static_cast<const __nv_bfloat16*>(gate_z);
+    opt.norm_w = norm_weight;
+    opt.norm_eps = norm_eps;
+    return launch_lean(a, ws.ptr, ws.bytes, reinterpret_cast<cudaStream_t>(stream), opt);
+}
+
 size_t gdn_workspace_bytes(int B, int T, int H, int d_k, int d_v, int packed) {
     return lean_workspace_bytes(B, T, H, d_k, d_v, packed != 0);
 }

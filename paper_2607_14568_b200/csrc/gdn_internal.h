@@ -53,6 +53,10 @@ struct LeanOptions {
     bool raw = false;          // q, k are raw projections and log_alpha, beta pre-activations: the prepare
     float gate_scale = 1.f;    //   kernel L2-normalises q, k and applies -softplus(.) * gate_scale and sigmoid(.)
     float eps = 0.f;           //   (eps under the square root of the norms)
+    // fused output stage (d_v = 128): out = o / sqrt(mean o^2 + norm_eps) * norm_w * silu(gate_z); nullptr = plain output
+    const __nv_bfloat16* gate_z = nullptr;
+    const float* norm_w = nullptr;
+    float norm_eps = 0.f;
 };
 int launch_lean(const PrefillArgs& a, void* workspace, size_t workspace_bytes, cudaStream_t stream,
                 const LeanOptions& opt = LeanOptions());

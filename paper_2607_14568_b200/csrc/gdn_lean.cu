@@ -216,7 +216,6 @@ gdn_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     uint8_t* sm = smem_raw + (base - smem_u32(smem_raw));
     float* sA = reinterpret_cast<float*>(sm + PS_A);
     float* sTf = sA;       // the solve overwrites A block by block
-    float* sY = reinterpret_cast<float*>(sm + PS_Y);
     float* gates = reinterpret_cast<float*>(sm + PS_GATES);
     float* sRN = reinterpret_cast<float*>(sm + PS_RN);
     volatile uint32_t* sMisc = reinterpret_cast<volatile uint32_t*>(sm + PS_MISC);
@@ -670,6 +669,10 @@ struct ChainParams {
     float* snaps;             // optional [B, nsnap, H, d_k, d_v]: the state after every snap_every chunks
     int snap_every, nsnap;
     int l2;                   // 1: the K, Q, V tiles are read for the last time here: mark them first to be evicted
+    // optional fused output stage (d_v = 128): out = o / sqrt(mean_j o_j^2 + norm_eps) * norm_w * silu(gate_z)
+    const __nv_bfloat16* gate_z;   // [.., H, d_v] like out, or nullptr
+    const float* norm_w;           // [d_v]
+    float norm_eps;
 };
 
 // One CTA's identity inside a kernel: aligned shared-memory base (address and pointer), tensor-memory base,
@@ -720,7 +723,7 @@ __device__ __forceinline__ void chain_init_bars(const Waiter& w) {
 
 // Steps c and d for one CTA.  SCAN: called from the merged scan kernel (register budgets are set there, the
 // incoming state is awaited through `hv` and read past the L1 cache, since another SM wrote it in this launch).
-template <bool DBG, bool SCAN>
+template <bool DBG, bool SCAN, bool GATED>
 __device__ __forceinline__ void chain_body(const CUtensorMap* map_q, const CUtensorMap* map_k, const CUtensorMap* map_v,
                                            const ChainParams& p, const Cta& cta, const Waiter& w, const Handover& hv) {
     const uint32_t base = cta.base, tmem = cta.tmem;
@@ -876,6 +879,55 @@ __device__ __forceinline__ void chain_body(const CUtensorMap* map_q, const CUten
             tmem_wait_ld();
             tc_fence_before_sync();
             mbar_arrive(w.bar(CB_OFREE));
+            if (GATED) {
+                // Fused output stage (the per-position kernels behind the scan, Section "Prefill projections:
+                // dequantize, then call the vendor"): root-mean-square norm of each output row over the value
+                // axis, weight vector, SiLU gate.  The rows go through shared memory in fp32, 32 tokens at a
+                // time; sixteen neighbouring lanes hold one row and add up its squares by shuffles.
+                float* fst = reinterpret_cast<float*>(sm + CS_OST);           // [32][128] fp32, the same 16 KiB
+                const size_t row0 = (size_t)(tok0 + c * C) * H + h;
+                const int col = (j & 15) * 8;
+                const float4 w0 = __ldg(reinterpret_cast<const float4*>(p.norm_w + col));
+                const float4 w1 = __ldg(reinterpret_cast<const float4*>(p.norm_w + col + 4));
+                const float wv[8] = {w0.x, w0.y, w0.z, w0.w, w1.x, w1.y, w1.z, w1.w};
+#pragma unroll
+                for (int half = 0; half < 2; ++half) {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i)
+                        fst[i * DVB + j] = half ? fmaf(gates[160 + i], __uint_as_float(o1b[i]), __uint_as_float(o2b[i]))
+                                                : fmaf(gates[128 + i], __uint_as_float(o1a[i]), __uint_as_float(o2a[i]));
+                    named_bar_sync(2, 128);
+#pragma unroll
+                    for (int it = 0; it < 4; ++it) {
+                        const int rr = (it * 128 + j) >> 4, r = 32 * half + rr;
+                        const float4 x0 = *reinterpret_cast<const float4*>(fst + rr * DVB + col);
+                        const float4 x1 = *reinterpret_cast<const float4*>(fst + rr * DVB + col + 4);
+                        const float xv[8] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w};
+                        float ss = 0.f;
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) ss = fmaf(xv[e], xv[e], ss);
+#pragma unroll
+                        for (int d = 1; d < 16; d <<= 1) ss += __shfl_xor_sync(0xffffffffu, ss, d);
+                        const float inv = rsqrtf(ss * (1.0f / DVB) + p.norm_eps);
+                        if (r < R) {
+                            const size_t off = (row0 + (size_t)r * H) * dv + col;
+                            const uint4 zz = *reinterpret_cast<const uint4*>(p.gate_z + off);
+                            const uint32_t zu[4] = {zz.x, zz.y, zz.z, zz.w};
+                            uint32_t pk[4];
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) {
+                                const float z0 = __uint_as_float(zu[e] << 16), z1 = __uint_as_float(zu[e] & 0xffff0000u);
+                                const float y0 = xv[2 * e] * inv * wv[2 * e] * (z0 / (1.0f + __expf(-z0)));
+                                const float y1 = xv[2 * e + 1] * inv * wv[2 * e + 1] * (z1 / (1.0f + __expf(-z1)));
+                                pk[e] = pack_bf16(y0, y1);
+                            }
+                            *reinterpret_cast<uint4*>(p.out + off) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                        }
+                    }
+                    named_bar_sync(2, 128);
+                }
+                continue;
+            }
 #pragma unroll
             for (int i = 0; i < 32; ++i) {
                 const float oa = fmaf(gates[128 + i], __uint_as_float(o1a[i]), __uint_as_float(o2a[i]));
@@ -1023,7 +1075,7 @@ __device__ __forceinline__ void chain_body(const CUtensorMap* map_q, const CUten
     }
 }
 
-template <bool DBG>
+template <bool DBG, bool GATED>
 __global__ void __launch_bounds__(CHAIN_THREADS, 1)
 gdn_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                  const __grid_constant__ CUtensorMap map_v, ChainParams p) {
@@ -1048,7 +1100,7 @@ gdn_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     const uint32_t tmem = sMisc[0];
     pdl_wait();                         // scratch items and incoming states come from the kernels before this one
     const Cta cta{base, sm, tmem, (int)blockIdx.x, (int)blockIdx.y, (int)blockIdx.z};
-    chain_body<DBG, false>(&map_q, &map_k, &map_v, p, cta, w, Handover{nullptr, 0});
+    chain_body<DBG, false, GATED>(&map_q, &map_k, &map_v, p, cta, w, Handover{nullptr, 0});
     tc_fence_before_sync();
     __syncthreads();
     if (warp == 0) {
@@ -1626,7 +1678,7 @@ gdn_scan_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         stamp(3);
         // ---------------- phase 3: chain over this segment's chunks ----------------
         const Cta c3{base, sm, tmem, 0, h, (int)blockIdx.z};
-        chain_body<DBG, true>(&map_q, &map_k, &map_v, p.cp, c3, w3, Handover{fl + 1, nowners});
+        chain_body<DBG, true, false>(&map_q, &map_k, &map_v, p.cp, c3, w3, Handover{fl + 1, nowners});
         stamp(4);
         tc_fence_before_sync();
         cta_sync();
@@ -1737,8 +1789,9 @@ static int device_setup(int* sms_out) {
         if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) return GDN_ERR_CUDA;
         if (cudaFuncSetAttribute(gdn_prep_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)PREP_SMEM) != cudaSuccess ||
             cudaFuncSetAttribute(gdn_prep_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)PREP_SMEM) != cudaSuccess ||
-            cudaFuncSetAttribute(gdn_chain_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)CHAIN_SMEM) != cudaSuccess ||
-            cudaFuncSetAttribute(gdn_chain_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)CHAIN_SMEM) != cudaSuccess ||
+            cudaFuncSetAttribute(gdn_chain_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)CHAIN_SMEM) != cudaSuccess ||
+            cudaFuncSetAttribute(gdn_chain_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)CHAIN_SMEM) != cudaSuccess ||
+            cudaFuncSetAttribute(gdn_chain_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)CHAIN_SMEM) != cudaSuccess ||
             cudaFuncSetAttribute(gdn_summary_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SUM_SMEM) != cudaSuccess ||
             cudaFuncSetAttribute(gdn_combine_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)CMB_SMEM) != cudaSuccess ||
             cudaFuncSetAttribute(gdn_scan_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SCAN_SMEM) != cudaSuccess ||
@@ -1755,6 +1808,7 @@ int launch_lean(const PrefillArgs& a, void* workspace, size_t workspace_bytes, c
     float* const snaps = opt.snaps;
     const int snap_every = opt.snap_every;
     if (!tc_supported(a.d_k, a.d_v)) return GDN_ERR_UNSUPPORTED;
+    if (opt.gate_z && a.d_v != DVB) return GDN_ERR_UNSUPPORTED;      // the fused norm sees one CTA's 128 value columns
     if (a.H > 65535 || a.B > 4095) return GDN_ERR_UNSUPPORTED;
     const bool packed = a.cu_seqlens != nullptr;
     const uint64_t tokens = packed ? (uint64_t)a.T : (uint64_t)a.B * a.T;
@@ -1814,10 +1868,10 @@ int launch_lean(const PrefillArgs& a, void* workspace, size_t workspace_bytes, c
         SummaryParams sp{a.cu_seqlens, ws, seg_n, seg_mt, a.B, a.T, a.H, a.d_v, nseg, seg_chunks, l2};
         CombineParams cb{a.initial_state, seg_n, seg_mt, seg_sin, a.H, a.d_v, nseg};
         // one resident CTA per (sequence, head, segment) runs all three phases when the grid fits the GPU at once
-        if (g_lean_use_scan && a.d_v == DVB && (long)a.B * a.H * nseg <= num_sms && (long)a.B * a.H <= kMaxScanChains) {
+        if (g_lean_use_scan && !opt.gate_z && a.d_v == DVB && (long)a.B * a.H * nseg <= num_sms && (long)a.B * a.H <= kMaxScanChains) {
             ChainParams cp{a.initial_state, static_cast<__nv_bfloat16*>(a.out), a.final_state, a.cu_seqlens,
                            ws, seg_sin, g_lean_dbg, g_lean_drop_chunk, a.B, a.T, a.H, a.d_v, nseg, seg_chunks,
-                           snaps, snap_every, nsnap, l2};
+                           snaps, snap_every, nsnap, l2, opt.gate_z, opt.norm_w, opt.norm_eps};
             ScanParams scp{sp, cb, cp, static_cast<int*>(workspace) + kScanFlagOffset};
             dim3 grid(1, a.H, a.B * nseg);
             if (g_lean_dbg) launch_after(gdn_scan_kernel<true>, grid, SCAN_THREADS, SCAN_SMEM, stream, mq, mk, mv, scp);
@@ -1841,10 +1895,11 @@ int launch_lean(const PrefillArgs& a, void* workspace, size_t workspace_bytes, c
     // ---- steps c, d ----
     ChainParams cp{a.initial_state, static_cast<__nv_bfloat16*>(a.out), a.final_state, a.cu_seqlens,
                    ws, seg_sin, g_lean_dbg, g_lean_drop_chunk, a.B, a.T, a.H, a.d_v, nseg, seg_chunks,
-                   snaps, snap_every, nsnap, l2};
+                   snaps, snap_every, nsnap, l2, opt.gate_z, opt.norm_w, opt.norm_eps};
     dim3 grid(a.d_v / DVB, a.H, a.B * nseg);
-    if (g_lean_dbg) launch_after(gdn_chain_kernel<true>, grid, CHAIN_THREADS, CHAIN_SMEM, stream, mq, mk, mv, cp);
-    else launch_after(gdn_chain_kernel<false>, grid, CHAIN_THREADS, CHAIN_SMEM, stream, mq, mk, mv, cp);
+    if (opt.gate_z) launch_after(gdn_chain_kernel<false, true>, grid, CHAIN_THREADS, CHAIN_SMEM, stream, mq, mk, mv, cp);
+    else if (g_lean_dbg) launch_after(gdn_chain_kernel<true, false>, grid, CHAIN_THREADS, CHAIN_SMEM, stream, mq, mk, mv, cp);
+    else launch_after(gdn_chain_kernel<false, false>, grid, CHAIN_THREADS, CHAIN_SMEM, stream, mq, mk, mv, cp);
     count_launch();
     mark(4);
     return cudaGetLastError() == cudaSuccess ? GDN_OK : GDN_ERR_CUDA;
@@ -1932,7 +1987,7 @@ int launch_lean_static(const PrefillArgs& a, cudaStream_t stream) {
             return GDN_ERR_CUDA;
         if (cudaFuncSetAttribute(gdn_prep_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)PREP_SMEM) != cudaSuccess ||
         cudaFuncSetAttribute(gdn_prep_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)PREP_SMEM) != cudaSuccess ||
-            cudaFuncSetAttribute(gdn_chain_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)CHAIN_SMEM) != cudaSuccess)
+            cudaFuncSetAttribute(gdn_chain_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)CHAIN_SMEM) != cudaSuccess)
             return GDN_ERR_CUDA;
         sms_of_device[dev] = sms;
         scratch_of_device[dev] = ptr;
@@ -1953,7 +2008,7 @@ int launch_lean_static(const PrefillArgs& a, cudaStream_t stream) {
                    ws, nullptr, nullptr, -1, a.B, a.T, a.H, a.d_v, 1, packed ? (1 << 24) : (nch > 0 ? nch : 1),
                    nullptr, 1, 0};
     dim3 grid(a.d_v / DVB, a.H, a.B);
-    gdn_chain_kernel<false><<<grid, CHAIN_THREADS, CHAIN_SMEM, stream>>>(mq, mk, mv, cp);
+    gdn_chain_kernel<false, false><<<grid, CHAIN_THREADS, CHAIN_SMEM, stream>>>(mq, mk, mv, cp);
     count_launch();
     return cudaGetLastError() == cudaSuccess ? GDN_OK : GDN_ERR_CUDA;
 }

@@ -202,3 +202,13 @@ def make_inputs(cfg: GdnConfig, threads: int = 8) -> GdnInputs:
         for nh in range(N * H):
             fill(nh)
     return GdnInputs(cfg, q, k, v, la, be, s0, cu, lengths)
+
+
+def epilogue_inputs(cfg: GdnConfig, lead_shape) -> Dict[str, np.ndarray]:
+    """Inputs of the fused output stage for a workload: the gate tensor z ~ N(0,1) with the shape of `out`
+    (``lead_shape + (H, d_v)``, stored like v) and the norm weight 1 + 0.1 N(0,1), fp32 [d_v].  One Philox
+    stream keyed by the seed and a constant no chain uses."""
+    rng = np.random.Generator(np.random.Philox(key=[cfg.seed, (1 << 40) + 17]))
+    z = rng.standard_normal(tuple(lead_shape) + (cfg.H, cfg.d_v), dtype=np.float32)
+    w = (1.0 + 0.1 * rng.standard_normal(cfg.d_v, dtype=np.float32)).astype(np.float32)
+    return {"z": _store(z, cfg.dtype), "weight": w}
