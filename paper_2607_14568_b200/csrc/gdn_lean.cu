@@ -67,10 +67,26 @@ constexpr uint32_t ITEM_BYTES = 34048;
 
 constexpr uint32_t LDA = 68, LDY = 32;
 
+// Bounded waits.  Their slow path is inlined at some thirty sites of kernels whose warp roles all run their
+// loops at once, and the instruction footprint decides the chain kernel's speed (measured: with 82 KiB of code
+// it ran at a 58 % instruction-cache hit rate and took 87 us on the 10240-token workload where 66 KiB took
+// 51 us), so the slow path is a counted loop: every pass suspends the thread for up to a millisecond, 1024
+// passes give the bound of about a second.  (An out-of-line function is not an option next to setmaxnreg.)
+constexpr uint32_t WAIT_PASS_NS = 1000000u;
+constexpr int WAIT_PASSES = 1024;
 struct Waiter {
     uint32_t bars;              // shared address of barrier 0
     volatile int* abort_flag;
     __device__ __forceinline__ uint32_t bar(uint32_t i) const { return bars + i * 8; }
+    __device__ __forceinline__ void wait_slow(uint32_t b, uint32_t parity) const {
+#pragma unroll 1
+        for (int i = 0; i < WAIT_PASSES; ++i) {
+            if (mbar_try_wait_suspend(b, parity, WAIT_PASS_NS)) return;
+            if (*abort_flag) return;
+        }
+        *abort_flag = 1;
+        atomicCAS(&g_lean_status, 0, (int)GDN_ERR_TIMEOUT);
+    }
     // For waits on the sequential chain: poll without suspending for a short while (a suspended
     // thread wakes up late), then fall back to the bounded suspending wait.
     __device__ __forceinline__ void wait_hot(uint32_t idx, uint32_t parity) const {
@@ -78,21 +94,12 @@ struct Waiter {
 #pragma unroll 1
         for (int i = 0; i < 4096; ++i)
             if (mbar_try_wait(b, parity)) return;
-        wait(idx, parity);
+        wait_slow(b, parity);
     }
     __device__ __forceinline__ void wait(uint32_t idx, uint32_t parity) const {
         const uint32_t b = bar(idx);
         if (mbar_try_wait(b, parity)) return;
-        const unsigned long long t0 = globaltimer_ns();
-        while (true) {
-            if (mbar_try_wait_suspend(b, parity, 100000u)) return;
-            if (*abort_flag) return;
-            if (globaltimer_ns() - t0 > TIMEOUT_NS) {
-                *abort_flag = 1;
-                atomicCAS(&g_lean_status, 0, (int)GDN_ERR_TIMEOUT);
-                return;
-            }
-        }
+        wait_slow(b, parity);
     }
 };
 
@@ -541,16 +548,11 @@ gdn_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             // ================= TMA + MMA issue (one thread) =================
             if (lane == 0) {
                 const uint32_t kq = base + PS_KQ, full = w.bar(PB_FULL);
-                const uint64_t pol_keep = l2_policy_evict_last();
+                const uint64_t pol_k = p.l2 ? l2_policy_evict_last() : l2_policy_evict_normal();
                 auto load_tiles = [&](int hh, long tk) {
                     mbar_arrive_expect_tx(full, 32768);
-                    if (p.l2) {
-                        tma_load_3d_hint(kq, &map_k, 0, hh, (int)tk, full, pol_keep);
-                        tma_load_3d_hint(kq + 16384, &map_k, 64, hh, (int)tk, full, pol_keep);
-                    } else {
-                        tma_load_3d(kq, &map_k, 0, hh, (int)tk, full);
-                        tma_load_3d(kq + 16384, &map_k, 64, hh, (int)tk, full);
-                    }
+                    tma_load_3d_hint(kq, &map_k, 0, hh, (int)tk, full, pol_k);
+                    tma_load_3d_hint(kq + 16384, &map_k, 64, hh, (int)tk, full, pol_k);
                     tma_load_3d(kq + 8192, &map_q, 0, hh, (int)tk, full);
                     tma_load_3d(kq + 24576, &map_q, 64, hh, (int)tk, full);
                 };
@@ -987,44 +989,51 @@ __device__ __forceinline__ void chain_body(const CUtensorMap* map_q, const CUten
             }
         } else if (warp == 10 && lane == 0) {
             // ---- MMA issuer of everything off the chain: U^T, O1^T, O2^T ----
-            auto issue_U = [&](int c) {                         // U^T = V^T (T diag(b))^T of chunk c
-                const uint32_t sB = c % 3, bb = base + CS_B + sB * STAGE_B;
-                w.wait(CB_FULLB0 + sB, (c / 3) & 1);
+            // (descriptors are built once; a stage or a k-step is an add on the 16-byte address field.  Every warp
+            //  role runs its loop at the same time, so the size of these loops shows in the instruction cache.)
+            const uint64_t dV0 = make_smem_desc(base + CS_B + ST_V, 8192, 1024), dT0 = make_smem_desc(base + CS_B + ST_T2, 1024, 1024);
+            const uint64_t dQ0 = make_smem_desc(base + CS_A + ST_KQ + 8192, 16, 1024), dP0 = make_smem_desc(base + CS_A + ST_P, 16, 1024);
+            for (int c = -1; c < nchunks; ++c) {
+                const uint32_t s = c & 1;
+                const uint64_t soff = (uint64_t)((s * STAGE_A) >> 4);
+                if (c >= 0) {
+                    w.wait(CB_SREADY, c & 1);
+                    w.wait(CB_FULLA0 + s, (c >> 1) & 1);
+                    if (c > 0) w.wait(CB_OFREE, (c - 1) & 1);  // the epilogue has read the previous O1, O2
+                    w.wait_hot(CB_V, c & 1);                   // stay out of the tensor pipe until v_new is done
+                    tc_fence_after_sync();
 #pragma unroll
-                for (uint32_t ks = 0; ks < 4; ++ks)
-                    mma_ss(tmem + TM_DV, make_smem_desc(bb + ST_V + ks * 2048, 8192, 1024),
-                           make_smem_desc(bb + ST_T2 + ks * 2048, 1024, 1024), ID_WU, ks > 0);
-                mma_commit(w.bar(CB_FREEB0 + sB));
-                mma_commit(w.bar(CB_U));
-            };
-            if (nchunks > 0) issue_U(0);
-            for (int c = 0; c < nchunks; ++c) {
-                const uint32_t s = c & 1, sb = base + CS_A + s * STAGE_A;
-                w.wait(CB_SREADY, c & 1);
-                w.wait(CB_FULLA0 + s, (c >> 1) & 1);
-                if (c > 0) w.wait(CB_OFREE, (c - 1) & 1);      // the epilogue has read the previous O1, O2
-                w.wait_hot(CB_V, c & 1);                       // stay out of the tensor pipe until v_new is done
-                tc_fence_after_sync();
+                    for (uint32_t ks = 0; ks < 8; ++ks)        // O1^T = S^T Q^T
+                        mma_ts(tmem + TM_O1, tmem + TM_SBF + ks * 8, dQ0 + soff + (uint64_t)(((ks >> 2) * 16384 + (ks & 3) * 32) >> 4),
+                               ID_O, ks > 0);
+                    mma_commit(w.bar(CB_O1));
+                    w.wait(CB_VREADY, c & 1);
+                    tc_fence_after_sync();
+                }
+                if (c + 1 < nchunks) {                         // U^T = V^T (T diag(b))^T of chunk c + 1: D_v is free,
+                    const uint32_t sB = (c + 1) % 3;           // v_new of chunk c has been read
+                    const uint64_t boff = (uint64_t)((sB * STAGE_B) >> 4);
+                    w.wait(CB_FULLB0 + sB, ((c + 1) / 3) & 1);
 #pragma unroll
-                for (uint32_t ks = 0; ks < 8; ++ks)            // O1^T = S^T Q^T
-                    mma_ts(tmem + TM_O1, tmem + TM_SBF + ks * 8,
-                           make_smem_desc(sb + ST_KQ + 8192 + (ks >> 2) * 16384 + (ks & 3) * 32, 16, 1024), ID_O, ks > 0);
-                mma_commit(w.bar(CB_O1));
-                w.wait(CB_VREADY, c & 1);
-                tc_fence_after_sync();
-                if (c + 1 < nchunks) issue_U(c + 1);           // D_v is free: v_new of chunk c has been read
+                    for (uint32_t ks = 0; ks < 4; ++ks)
+                        mma_ss(tmem + TM_DV, dV0 + boff + ks * 128, dT0 + boff + ks * 128, ID_WU, ks > 0);
+                    mma_commit(w.bar(CB_FREEB0 + sB));
+                    mma_commit(w.bar(CB_U));
+                }
+                if (c >= 0) {
 #pragma unroll
-                for (uint32_t ks = 0; ks < 4; ++ks)            // O2^T = v^T P^T
-                    mma_ts(tmem + TM_O2, tmem + TM_V + ks * 8, make_smem_desc(sb + ST_P + ks * 32, 16, 1024), ID_O, ks > 0);
-                mma_commit(w.bar(CB_O));
-                mma_commit(w.bar(CB_FREEA0 + s));
+                    for (uint32_t ks = 0; ks < 4; ++ks)        // O2^T = v^T P^T
+                        mma_ts(tmem + TM_O2, tmem + TM_V + ks * 8, dP0 + soff + ks * 2, ID_O, ks > 0);
+                    mma_commit(w.bar(CB_O));
+                    mma_commit(w.bar(CB_FREEA0 + s));
+                }
             }
         } else if (warp == 9 && lane == 0) {
             // ---- TMA producer ----
             prefetch_tensormap(map_q);
             prefetch_tensormap(map_k);
             prefetch_tensormap(map_v);
-            const uint64_t pol_done = l2_policy_evict_first();
+            const uint64_t pol_done = p.l2 ? l2_policy_evict_first() : l2_policy_evict_normal();
             for (int c = 0; c < nchunks; ++c) {
                 if (c == p.drop_chunk && dvb == 0 && h == 0 && cta.z == 0) continue;
                 const int tok = (int)(tok0 + (long)c * C);
@@ -1033,13 +1042,8 @@ __device__ __forceinline__ void chain_body(const CUtensorMap* map_q, const CUten
                     const uint32_t sB = c % 3, bb = base + CS_B + sB * STAGE_B, full = w.bar(CB_FULLB0 + sB);
                     if (c >= 3) w.wait(CB_FREEB0 + sB, ((c / 3) - 1) & 1);
                     mbar_arrive_expect_tx(full, STAGE_B_TX);
-                    if (p.l2) {
-                        tma_load_3d_hint(bb + ST_V, map_v, dvb * DVB, h, tok, full, pol_done);
-                        tma_load_3d_hint(bb + ST_V + 8192, map_v, dvb * DVB + 64, h, tok, full, pol_done);
-                    } else {
-                        tma_load_3d(bb + ST_V, map_v, dvb * DVB, h, tok, full);
-                        tma_load_3d(bb + ST_V + 8192, map_v, dvb * DVB + 64, h, tok, full);
-                    }
+                    tma_load_3d_hint(bb + ST_V, map_v, dvb * DVB, h, tok, full, pol_done);
+                    tma_load_3d_hint(bb + ST_V + 8192, map_v, dvb * DVB + 64, h, tok, full, pol_done);
                     bulk_load(bb + ST_T2, item + IT_T2, 8192, full);
                 }
                 {   // ring A: K/Q tiles, -W^T, P, and the gate vectors (own 4-deep ring, same barrier)
@@ -1047,17 +1051,10 @@ __device__ __forceinline__ void chain_body(const CUtensorMap* map_q, const CUten
                     if (c >= 2) w.wait(CB_FREEA0 + s, ((c >> 1) - 1) & 1);
                     mbar_arrive_expect_tx(full, STAGE_A_TX);
                     bulk_load(sb + ST_W, item + IT_W, 16384, full);
-                    if (p.l2) {
-                        tma_load_3d_hint(sb + ST_KQ, map_k, 0, h, tok, full, pol_done);
-                        tma_load_3d_hint(sb + ST_KQ + 8192, map_q, 0, h, tok, full, pol_done);
-                        tma_load_3d_hint(sb + ST_KQ + 16384, map_k, 64, h, tok, full, pol_done);
-                        tma_load_3d_hint(sb + ST_KQ + 24576, map_q, 64, h, tok, full, pol_done);
-                    } else {
-                        tma_load_3d(sb + ST_KQ, map_k, 0, h, tok, full);
-                        tma_load_3d(sb + ST_KQ + 8192, map_q, 0, h, tok, full);
-                        tma_load_3d(sb + ST_KQ + 16384, map_k, 64, h, tok, full);
-                        tma_load_3d(sb + ST_KQ + 24576, map_q, 64, h, tok, full);
-                    }
+                    tma_load_3d_hint(sb + ST_KQ, map_k, 0, h, tok, full, pol_done);
+                    tma_load_3d_hint(sb + ST_KQ + 8192, map_q, 0, h, tok, full, pol_done);
+                    tma_load_3d_hint(sb + ST_KQ + 16384, map_k, 64, h, tok, full, pol_done);
+                    tma_load_3d_hint(sb + ST_KQ + 24576, map_q, 64, h, tok, full, pol_done);
                     bulk_load(sb + ST_P, item + IT_P, 8192, full);
                     bulk_load(base + CS_GATES + (c & 3) * 1280, item + IT_GATES, 1280, full);
                 }
@@ -1312,7 +1309,7 @@ __device__ __forceinline__ void summary_body(const CUtensorMap* map_k, const CUt
         } else if (warp == 9 && lane == 0) {
             prefetch_tensormap(map_k);
             prefetch_tensormap(map_v);
-            const uint64_t pol_keep = l2_policy_evict_last();
+            const uint64_t pol_keep = p.l2 ? l2_policy_evict_last() : l2_policy_evict_normal();
             for (int c = 0; c < nchunks; ++c) {
                 const uint32_t s = c % SUM_STAGES, sb = base + s * SUM_STAGE;
                 if (c >= (int)SUM_STAGES) w.wait(SB_FREE0 + s, ((c / SUM_STAGES) - 1) & 1);
@@ -1320,17 +1317,10 @@ __device__ __forceinline__ void summary_body(const CUtensorMap* map_k, const CUt
                 const int tok = (int)(tok0 + (long)c * C);
                 const uint8_t* item = p.items + (size_t)((slot0 + c) * H + h) * ITEM_BYTES;
                 mbar_arrive_expect_tx(full, SUM_STAGE_TX);
-                if (p.l2) {
-                    tma_load_3d_hint(sb + SS_K, map_k, 0, h, tok, full, pol_keep);
-                    tma_load_3d_hint(sb + SS_K + 8192, map_k, 64, h, tok, full, pol_keep);
-                    tma_load_3d_hint(sb + SS_V, map_v, dvb * DVB, h, tok, full, pol_keep);
-                    tma_load_3d_hint(sb + SS_V + 8192, map_v, dvb * DVB + 64, h, tok, full, pol_keep);
-                } else {
-                    tma_load_3d(sb + SS_K, map_k, 0, h, tok, full);
-                    tma_load_3d(sb + SS_K + 8192, map_k, 64, h, tok, full);
-                    tma_load_3d(sb + SS_V, map_v, dvb * DVB, h, tok, full);
-                    tma_load_3d(sb + SS_V + 8192, map_v, dvb * DVB + 64, h, tok, full);
-                }
+                tma_load_3d_hint(sb + SS_K, map_k, 0, h, tok, full, pol_keep);
+                tma_load_3d_hint(sb + SS_K + 8192, map_k, 64, h, tok, full, pol_keep);
+                tma_load_3d_hint(sb + SS_V, map_v, dvb * DVB, h, tok, full, pol_keep);
+                tma_load_3d_hint(sb + SS_V + 8192, map_v, dvb * DVB + 64, h, tok, full, pol_keep);
                 bulk_load(sb + SS_W, item + IT_W, 16384, full);
                 bulk_load(sb + SS_T2, item + IT_T2, 8192, full);
                 bulk_load(sb + SS_GATES, item + IT_GATES, 1280, full);
