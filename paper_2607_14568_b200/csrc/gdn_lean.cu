@@ -341,7 +341,9 @@ gdn_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
 #pragma unroll
                                 for (int e = 0; e < 4; ++e) {
                                     const int i = 32 * hh + 4 * i4 + e;
-                                    o[e] = (i < r) ? br * y[4 * i4 + e] : 0.f;
+                                    // rows of padded tokens (r >= R) by select too: their K rows are whatever follows the
+                                    // sequence in memory, possibly not finite, and 0 * NaN would spread through the merges
+                                    o[e] = (i < r && r < R) ? br * y[4 * i4 + e] : 0.f;
                                 }
                                 st_shared_f4(base + PS_A + (r * LDA + 32 * hh + 4 * i4) * 4, o[0], o[1], o[2], o[3]);
                             }
@@ -362,6 +364,16 @@ gdn_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
 #pragma unroll
                         for (int ch = 0; ch < 4; ++ch) st_shared_v4(pimg + swz(r, 4 * hh + ch), 0u, 0u, 0u, 0u);
                     }
+                }
+            }
+            if (R < C) {
+                // Tail chunk: the tile rows behind the sequence's last token hold the first rows of whatever follows
+                // in memory.  They only ever meet factors that are exactly zero, but zero times a non-finite value
+                // is not zero: clear the K rows (the W product contracts over them) now that G has been formed.
+                const uint32_t pieces = (uint32_t)(C - R) * 8u;            // 16-byte pieces per 64-column half
+                for (uint32_t x = tp; x < 2 * pieces; x += 128) {
+                    const uint32_t half = x >= pieces ? 1u : 0u, y = x - half * pieces;
+                    st_shared_v4(base + PS_KQ + half * 16384 + ((uint32_t)R + (y >> 3)) * 128 + ((y & 7) << 4), 0u, 0u, 0u, 0u);
                 }
             }
             fence_proxy_async_smem();
@@ -654,7 +666,7 @@ constexpr uint32_t CS_TOTAL = CS_MISC + 64;
 constexpr uint32_t CHAIN_SMEM = CS_TOTAL + 1024;
 
 enum CBar : uint32_t { CB_FULLA0 = 0, CB_FREEA0 = 2, CB_FULLB0 = 4, CB_FREEB0 = 7, CB_V = 10, CB_S, CB_O, CB_SREADY, CB_VREADY, CB_OFREE,
-                       CB_U, CB_O1 };
+                       CB_U, CB_O1, CB_CLEAN };
 
 struct ChainParams {
     const float* s0;          // [N,H,d_k,d_v] or nullptr
@@ -721,6 +733,7 @@ __device__ __forceinline__ void chain_init_bars(const Waiter& w) {
     for (uint32_t i = 0; i < 3; ++i) { mbar_init(w.bar(CB_FULLB0 + i), 1); mbar_init(w.bar(CB_FREEB0 + i), 1); }
     mbar_init(w.bar(CB_V), 1); mbar_init(w.bar(CB_S), 1); mbar_init(w.bar(CB_O), 1);
     mbar_init(w.bar(CB_SREADY), 128); mbar_init(w.bar(CB_VREADY), 128); mbar_init(w.bar(CB_OFREE), 128);
+    mbar_init(w.bar(CB_CLEAN), 128);
 }
 
 // Steps c and d for one CTA.  SCAN: called from the merged scan kernel (register budgets are set there, the
@@ -741,6 +754,11 @@ __device__ __forceinline__ void chain_body(const CUtensorMap* map_q, const CUten
     const int len = max(0, min(sq.len - cbeg * C, p.seg_chunks * C));
     const int nchunks = (len + C - 1) / C;
     const long slot0 = slot_base(sq.tok0, n) + cbeg;
+    // A last chunk with fewer than 64 tokens: its K and V tile rows behind the last token hold the first rows of
+    // whatever follows the sequence in memory.  They only meet factors that are exactly zero, but zero times a
+    // non-finite value is not zero, so the epilogue warpgroup clears them once the tiles have landed and the MMAs
+    // that contract over tokens (U, the state update) wait for that (barrier CB_CLEAN, used once per CTA).
+    const int tail_c = (nchunks > 0 && (len & (C - 1)) != 0) ? nchunks - 1 : -1;
     const unsigned long long t_start = DBG ? globaltimer_ns() : 0ull;
     auto stamp = [&](int role, int c, int ev) {
         if (DBG && p.dbg && dvb == 0 && h == 0 && cta.z == 0 && c < 32)
@@ -869,6 +887,21 @@ __device__ __forceinline__ void chain_body(const CUtensorMap* map_q, const CUten
         for (int c = 0; c < nchunks; ++c) {
             const int R = min(C, len - c * C);
             const float* gates = reinterpret_cast<const float*>(sm + CS_GATES + (c & 3) * 1280);
+            if (tail_c >= 0 && c == max(tail_c - 1, 0)) {
+                const int Rt = len - tail_c * C;
+                const uint32_t sa = base + CS_A + (uint32_t)(tail_c & 1) * STAGE_A + ST_KQ;
+                const uint32_t sv = base + CS_B + (uint32_t)(tail_c % 3) * STAGE_B + ST_V;
+                w.wait(CB_FULLA0 + (tail_c & 1), (tail_c >> 1) & 1);
+                w.wait(CB_FULLB0 + tail_c % 3, (tail_c / 3) & 1);
+                const uint32_t pieces = (uint32_t)(C - Rt) * 8u;
+                for (uint32_t x = j; x < 4 * pieces; x += 128) {             // K_lo, K_hi, V_lo, V_hi
+                    const uint32_t t4 = x / pieces, y = x - t4 * pieces;
+                    const uint32_t tile = t4 == 0 ? sa : t4 == 1 ? sa + 16384 : t4 == 2 ? sv : sv + 8192;
+                    st_shared_v4(tile + ((uint32_t)Rt + (y >> 3)) * 128 + ((y & 7) << 4), 0u, 0u, 0u, 0u);
+                }
+                fence_proxy_async_smem();
+                mbar_arrive(w.bar(CB_CLEAN));
+            }
             w.wait_hot(CB_O, c & 1);
             tc_fence_after_sync();
             // take both accumulators out of tensor memory first and hand them back at once: the next
@@ -969,6 +1002,7 @@ __device__ __forceinline__ void chain_body(const CUtensorMap* map_q, const CUten
                 // state sits on the dependent chain
                 w.wait_hot(CB_FULLA0 + s, (c >> 1) & 1);
                 w.wait_hot(CB_U, c & 1);                       // U^T of this chunk is in the accumulator
+                if (c == tail_c) w.wait_hot(CB_CLEAN, 0);      // padded K rows have been cleared
                 w.wait_hot(CB_SREADY, c & 1);
                 tc_fence_after_sync();
                 stamp(1, c, 0);
@@ -1014,6 +1048,7 @@ __device__ __forceinline__ void chain_body(const CUtensorMap* map_q, const CUten
                     const uint32_t sB = (c + 1) % 3;           // v_new of chunk c has been read
                     const uint64_t boff = (uint64_t)((sB * STAGE_B) >> 4);
                     w.wait(CB_FULLB0 + sB, ((c + 1) / 3) & 1);
+                    if (c + 1 == tail_c) w.wait(CB_CLEAN, 0);  // padded V rows have been cleared
 #pragma unroll
                     for (uint32_t ks = 0; ks < 4; ++ks)
                         mma_ss(tmem + TM_DV, dV0 + boff + ks * 128, dT0 + boff + ks * 128, ID_WU, ks > 0);

@@ -332,6 +332,7 @@ gdn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
         const uint32_t lane_base = (uint32_t)(wp * 32) << 16;
         for (int c = 0; c < nchunks; ++c) {
             const uint32_t buf = c & 1;
+            const int Rc = min(C, len - c * C);                // valid tokens of this chunk
             const float* gates = sGates + (c & 3) * GATE_FLOATS;
             if (tp == 0) stamp(1, c, 0);
             wait(cta, B_GREADY0 + (c & 3), (c >> 2) & 1);      // step a runs ahead in its own warp
@@ -372,7 +373,8 @@ gdn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
 #pragma unroll
                                 for (int e = 0; e < 4; ++e) {
                                     const int i = 32 * hh + 4 * i4 + e;
-                                    o[e] = (i < r) ? br * y[4 * i4 + e] : 0.f;
+                                    // rows of padded tokens by select too (their K rows need not be finite)
+                                    o[e] = (i < r && r < Rc) ? br * y[4 * i4 + e] : 0.f;
                                 }
                                 st_shared_f4(cta.base + SM_A + (r * LDA + 32 * hh + 4 * i4) * 4, o[0], o[1], o[2], o[3]);
                             }
@@ -526,6 +528,18 @@ gdn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
                     }
                     st_shared_v4(cta.base + SM_T1 + swz(cc, 4 * half + ch), p1[0], p1[1], p1[2], p1[3]);
                     st_shared_v4(cta.base + SM_T2 + swz(cc, 4 * half + ch), p2[0], p2[1], p2[2], p2[3]);
+                }
+            }
+            if (Rc < C) {
+                // Tail chunk: the K and V tile rows behind the last token hold the first rows of whatever follows the
+                // sequence in memory.  They only meet factors that are exactly zero, but zero times a non-finite value
+                // is not zero: clear them before the products that contract over tokens (W, U, the state update).
+                const uint32_t kq = cta.base + SM_KQ + buf * 32768, vb = cta.base + SM_V + buf * 16384;
+                const uint32_t pieces = (uint32_t)(C - Rc) * 8u;
+                for (uint32_t x = tp; x < 4 * pieces; x += 128) {
+                    const uint32_t t4 = x / pieces, y = x - t4 * pieces;
+                    const uint32_t tile = t4 == 0 ? kq : t4 == 1 ? kq + 16384 : t4 == 2 ? vb : vb + 8192;
+                    st_shared_v4(tile + ((uint32_t)Rc + (y >> 3)) * 128 + ((y & 7) << 4), 0u, 0u, 0u, 0u);
                 }
             }
             fence_proxy_async_smem();

@@ -341,3 +341,23 @@ def test_error_codes():
     assert L.gdn_chunk_prefill(*args) == 0
     torch.cuda.synchronize()
     assert gdn.gdn_launch_count() > n0
+
+
+# ---- a ragged tail next to non-finite neighbours ----------------------------------------------------------
+@pytest.mark.parametrize("impl", ["fused", "two_kernel", "simt"])
+def test_bf16_tail_chunk_is_immune_to_what_follows_the_sequence(impl):
+    """Packed input: the tile rows behind a sequence's last token are the first rows of the next sequence.  They only
+    meet factors that are exactly zero, but 0 x inf is not 0 -- so the second sequence here starts with rows of inf
+    and NaN in q, k and v, and the first sequence (100 tokens: a 36-token tail chunk) must still come out as the
+    recurrence over its own tokens.  (The second sequence's own results are not finite, as they should be.)"""
+    cfg = get_config("serving", B=2, H=2, lengths=(100, 90), seed=99)
+    x = make_inputs(cfg)
+    bad = np.array([0x7F80, 0xFF80, 0x7FC0], dtype=np.uint16)            # +inf, -inf, NaN in bf16
+    for t in (x.q, x.k, x.v):
+        t[100:140] = bad[np.arange(t[100:140].size).reshape(t[100:140].shape) % 3]
+    d = to_device(x)
+    out, fin = run_lib(BF16_FNS[impl], d)
+    o_ref, f_ref = oracle.sequential(widen(x.q[None, :100]), widen(x.k[None, :100]), widen(x.v[None, :100]),
+                                     x.log_alpha[None, :100], x.beta[None, :100], x.initial_state[:1])
+    assert_close(f64(out[:100]), o_ref[0], BF16_REL_L2, BF16_MAX_ABS, impl + " first sequence out")
+    assert_close(f64(fin[0]), f_ref[0], BF16_REL_L2, BF16_MAX_ABS, impl + " first sequence final_state")
