@@ -314,7 +314,9 @@ gdn_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                 const bool is_a = tp < 64;
                 const int rmax = 32 * (warp & 1) + 31;
                 const uint32_t pimg = base + PS_KQ + 8192;   // the Q_lo sub-tile is dead once G is complete
-#pragma unroll
+                // (one copy of the 32-column body: four CTAs per SM sit in different phases of this kernel, so all of
+                //  its code is live at once and its size shows in the instruction cache)
+#pragma unroll 1
                 for (int hh = 0; hh < 2; ++hh) {
                     if (32 * hh <= rmax) {
                         uint32_t x[32];
@@ -419,7 +421,7 @@ gdn_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                 if (warp < 2) {   // level 1: the 16-blocks (1,0) and (3,2), one warp each
                     const int lo = 32 * warp, hi = lo + 16;
                     float z[2][4] = {};
-#pragma unroll
+#pragma unroll 1
                     for (int ks = 0; ks < 2; ++ks) {
                         const float2 a01 = *reinterpret_cast<const float2*>(sTf + (hi + g) * LDA + hi + 8 * ks + 2 * t);
                         const float2 a23 = *reinterpret_cast<const float2*>(sTf + (hi + g + 8) * LDA + hi + 8 * ks + 2 * t);
@@ -454,7 +456,7 @@ gdn_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                 // T11 starts at row 16.
                 const int mb = warp & 1, nb = warp >> 1;
                 float z[4][4] = {};
-#pragma unroll
+#pragma unroll 1
                 for (int ks = 0; ks < 4; ++ks) {
                     if (ks < 2 * (mb + 1)) {
                         const float2 a01 = *reinterpret_cast<const float2*>(sTf + (32 + 16 * mb + g) * LDA + 32 + 8 * ks + 2 * t);
