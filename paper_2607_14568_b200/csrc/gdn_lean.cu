@@ -41,7 +41,9 @@ static cudaEvent_t g_lean_events[5] = {nullptr, nullptr, nullptr, nullptr, nullp
 static bool g_lean_split_last = false;
 static float* g_lean_dbg = nullptr;        // debug: time stamps of the chain kernel
 static int g_lean_drop_chunk = -1;         // tests: chunk the chain kernel's TMA thread skips (-1 = none)
-static int g_lean_l2_hints = 1;            // tests: 0 = no L2 eviction-priority hints on the tile loads
+static int g_lean_l2_hints = 3;            // tests: bit 0 = L2 eviction-priority hints on the K, Q, V tile loads, bit 1 = on the
+                                           // scratch images W and T2 (measured on the 10240-token workload, chain kernel:
+                                           // 51.3 us without, 49.0 / 49.4 us with either, 47.2 us with both)
 static bool g_lean_use_scan = false;       // true = summary, combination and chain of a split run as one resident launch (measured
                                            // slower than the three kernels under programmatic dependent launch: 0.162 vs 0.152 ms on
                                            // the 10240-token workload, 0.074 vs 0.060 ms at 2048 tokens, so it is off by default)
@@ -138,6 +140,15 @@ __device__ __forceinline__ void bulk_store(void* gdst, uint32_t smem_src, uint32
     asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
                  ::"l"(reinterpret_cast<uint64_t>(gdst)), "r"(smem_src), "r"(bytes) : "memory");
 }
+// the same copies with an L2 eviction-priority hint
+__device__ __forceinline__ void bulk_load_hint(uint32_t smem_dst, const void* gsrc, uint32_t bytes, uint32_t bar, uint64_t pol) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
+                 ::"r"(smem_dst), "l"(reinterpret_cast<uint64_t>(gsrc)), "r"(bytes), "r"(bar), "l"(pol) : "memory");
+}
+__device__ __forceinline__ void bulk_store_hint(void* gdst, uint32_t smem_src, uint32_t bytes, uint64_t pol) {
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group.L2::cache_hint [%0], [%1], %2, %3;"
+                 ::"l"(reinterpret_cast<uint64_t>(gdst)), "r"(smem_src), "r"(bytes), "l"(pol) : "memory");
+}
 __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void bulk_wait_read_all() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
 __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
@@ -182,7 +193,8 @@ struct PrepParams {
     int B, T, H;
     float gate_scale, eps;     // raw inputs only
     int* ticket;               // {next item, CTAs done}: both zero before the launch, both zero again after it
-    int l2;                    // 1: the K tiles are read again by later kernels of this call and fit in L2: keep them there
+    int l2;                    // bit 0: the K tiles are read again by later kernels of this call and fit in L2: keep them there;
+                               // bit 1: the same for the W and T2 images this kernel writes
 };
 
 constexpr uint32_t ID_G = make_idesc(128, 64, kFmtBF16, kFmtBF16, kMajorK, kMajorK);
@@ -517,7 +529,7 @@ gdn_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             tc_fence_before_sync();
             mbar_arrive(w.bar(PB_TREADY));
             named_bar_sync(1, 128);
-            if (tp == 0) { bulk_store(out_item + IT_T2, base + PS_T2, 8192); bulk_commit(); }
+            if (tp == 0) { bulk_store_hint(out_item + IT_T2, base + PS_T2, 8192, (p.l2 & 2) ? l2_policy_evict_last() : l2_policy_evict_normal()); bulk_commit(); }
             // ---- step b3 result: -W^T image to scratch; gate vectors to scratch ----
             if (tp < GATE_FLOATS / 4) {
                 float4 gv = *reinterpret_cast<const float4*>(gates + 4 * tp);
@@ -552,7 +564,7 @@ gdn_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             fence_proxy_async_smem();
             named_bar_sync(1, 128);
             if (tp == 0) {                                     // staged over the fp32 T, which is dead by now
-                bulk_store(out_item + IT_W, base + PS_A, 16384);
+                bulk_store_hint(out_item + IT_W, base + PS_A, 16384, (p.l2 & 2) ? l2_policy_evict_last() : l2_policy_evict_normal());
                 bulk_commit();
                 bulk_wait_read_all();                          // the staging space may now be overwritten
             }
@@ -562,7 +574,7 @@ gdn_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             // ================= TMA + MMA issue (one thread) =================
             if (lane == 0) {
                 const uint32_t kq = base + PS_KQ, full = w.bar(PB_FULL);
-                const uint64_t pol_k = p.l2 ? l2_policy_evict_last() : l2_policy_evict_normal();
+                const uint64_t pol_k = (p.l2 & 1) ? l2_policy_evict_last() : l2_policy_evict_normal();
                 auto load_tiles = [&](int hh, long tk) {
                     mbar_arrive_expect_tx(full, 32768);
                     tma_load_3d_hint(kq, &map_k, 0, hh, (int)tk, full, pol_k);
@@ -684,7 +696,7 @@ struct ChainParams {
     int nseg, seg_chunks;     // segments per sequence (1 = no split) and chunks per segment
     float* snaps;             // optional [B, nsnap, H, d_k, d_v]: the state after every snap_every chunks
     int snap_every, nsnap;
-    int l2;                   // 1: the K, Q, V tiles are read for the last time here: mark them first to be evicted
+    int l2;                   // bit 0: the K, Q, V tiles are read for the last time here: mark them first to be evicted; bit 1: W, T2 too
     // optional fused output stage (d_v = 128): out = o / sqrt(mean_j o_j^2 + norm_eps) * norm_w * silu(gate_z)
     const __nv_bfloat16* gate_z;   // [.., H, d_v] like out, or nullptr
     const float* norm_w;           // [d_v]
@@ -1070,7 +1082,8 @@ __device__ __forceinline__ void chain_body(const CUtensorMap* map_q, const CUten
             prefetch_tensormap(map_q);
             prefetch_tensormap(map_k);
             prefetch_tensormap(map_v);
-            const uint64_t pol_done = p.l2 ? l2_policy_evict_first() : l2_policy_evict_normal();
+            const uint64_t pol_done = (p.l2 & 1) ? l2_policy_evict_first() : l2_policy_evict_normal();
+            const uint64_t pol_item = (p.l2 & 2) ? l2_policy_evict_first() : l2_policy_evict_normal();
             for (int c = 0; c < nchunks; ++c) {
                 if (c == p.drop_chunk && dvb == 0 && h == 0 && cta.z == 0) continue;
                 const int tok = (int)(tok0 + (long)c * C);
@@ -1081,13 +1094,13 @@ __device__ __forceinline__ void chain_body(const CUtensorMap* map_q, const CUten
                     mbar_arrive_expect_tx(full, STAGE_B_TX);
                     tma_load_3d_hint(bb + ST_V, map_v, dvb * DVB, h, tok, full, pol_done);
                     tma_load_3d_hint(bb + ST_V + 8192, map_v, dvb * DVB + 64, h, tok, full, pol_done);
-                    bulk_load(bb + ST_T2, item + IT_T2, 8192, full);
+                    bulk_load_hint(bb + ST_T2, item + IT_T2, 8192, full, pol_item);
                 }
                 {   // ring A: K/Q tiles, -W^T, P, and the gate vectors (own 4-deep ring, same barrier)
                     const uint32_t s = c & 1, sb = base + CS_A + s * STAGE_A, full = w.bar(CB_FULLA0 + s);
                     if (c >= 2) w.wait(CB_FREEA0 + s, ((c >> 1) - 1) & 1);
                     mbar_arrive_expect_tx(full, STAGE_A_TX);
-                    bulk_load(sb + ST_W, item + IT_W, 16384, full);
+                    bulk_load_hint(sb + ST_W, item + IT_W, 16384, full, pol_item);
                     tma_load_3d_hint(sb + ST_KQ, map_k, 0, h, tok, full, pol_done);
                     tma_load_3d_hint(sb + ST_KQ + 8192, map_q, 0, h, tok, full, pol_done);
                     tma_load_3d_hint(sb + ST_KQ + 16384, map_k, 64, h, tok, full, pol_done);
@@ -1182,7 +1195,7 @@ struct SummaryParams {
     float* seg_mt;            // [B*nseg, H] x 64 KiB: M_seg^T as two bf16 operand images (leading part | remainder)
     int B, T, H, dv;
     int nseg, seg_chunks;
-    int l2;                   // 1: K and V are read again by the chain phase and fit in L2: keep them there
+    int l2;                   // bit 0: K and V are read again by the chain phase and fit in L2: keep them there; bit 1: W, T2 too
 };
 
 __device__ __forceinline__ void summary_init_bars(const Waiter& w, int ninst) {
@@ -1346,7 +1359,8 @@ __device__ __forceinline__ void summary_body(const CUtensorMap* map_k, const CUt
         } else if (warp == 9 && lane == 0) {
             prefetch_tensormap(map_k);
             prefetch_tensormap(map_v);
-            const uint64_t pol_keep = p.l2 ? l2_policy_evict_last() : l2_policy_evict_normal();
+            const uint64_t pol_keep = (p.l2 & 1) ? l2_policy_evict_last() : l2_policy_evict_normal();
+            const uint64_t pol_item = (p.l2 & 2) ? l2_policy_evict_last() : l2_policy_evict_normal();
             for (int c = 0; c < nchunks; ++c) {
                 const uint32_t s = c % SUM_STAGES, sb = base + s * SUM_STAGE;
                 if (c >= (int)SUM_STAGES) w.wait(SB_FREE0 + s, ((c / SUM_STAGES) - 1) & 1);
@@ -1358,8 +1372,8 @@ __device__ __forceinline__ void summary_body(const CUtensorMap* map_k, const CUt
                 tma_load_3d_hint(sb + SS_K + 8192, map_k, 64, h, tok, full, pol_keep);
                 tma_load_3d_hint(sb + SS_V, map_v, dvb * DVB, h, tok, full, pol_keep);
                 tma_load_3d_hint(sb + SS_V + 8192, map_v, dvb * DVB + 64, h, tok, full, pol_keep);
-                bulk_load(sb + SS_W, item + IT_W, 16384, full);
-                bulk_load(sb + SS_T2, item + IT_T2, 8192, full);
+                bulk_load_hint(sb + SS_W, item + IT_W, 16384, full, pol_item);
+                bulk_load_hint(sb + SS_T2, item + IT_T2, 8192, full, pol_item);
                 bulk_load(sb + SS_GATES, item + IT_GATES, 1280, full);
             }
             if (*w.abort_flag) {
@@ -1872,7 +1886,7 @@ int launch_lean(const PrefillArgs& a, void* workspace, size_t workspace_bytes, c
     // ---- state-independent steps, every (chunk, head) ----
     // With a split, K (and V) are read by two or three kernels of the call; when they fit in L2 comfortably the
     // earlier readers ask L2 to keep them and the last reader releases them.
-    const int l2 = (g_lean_l2_hints && nseg > 1 && tokens * a.H * (uint64_t)(a.d_k + a.d_v) * 2 <= (96ull << 20)) ? 1 : 0;
+    const int l2 = (nseg > 1 && tokens * a.H * (uint64_t)(a.d_k + a.d_v) * 2 <= (96ull << 20)) ? (g_lean_l2_hints & 3) : 0;
     PrepParams pp{a.log_alpha, a.beta, a.cu_seqlens, ws, nslots, a.B, a.T, a.H, opt.gate_scale, opt.eps, ticket, l2};
     const int pgrid = (int)(nitems < 4L * num_sms ? nitems : 4L * num_sms);
     auto mark = [&](int i) { if (g_lean_timing && g_lean_events[i]) cudaEventRecord(g_lean_events[i], stream); };
