@@ -484,6 +484,18 @@ def run_attention(args):
                                    "kernel": "attn_causal_kernel", "algorithmic_flops": flops}}), flush=True)
 
 
+def replica_launch_command(n_gpus, argv, port=None):
+    """The command that starts `n_gpus` replica processes of this script on one node (one rank per GPU,
+    rendezvous on 127.0.0.1), as the driver's launcher would."""
+    if port is None:
+        import socket
+        with socket.socket() as sk:
+            sk.bind(("127.0.0.1", 0))
+            port = sk.getsockname()[1]
+    return [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n_gpus}",
+            "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + list(argv)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -496,13 +508,7 @@ def main():
     args = ap.parse_args()
     if args.gpus > 1 and "WORLD_SIZE" not in os.environ and args.impl == "ours":
         # not started by a launcher: start one replica process per GPU ourselves (rank 0 prints the line)
-        import socket
-        with socket.socket() as sk:
-            sk.bind(("127.0.0.1", 0))
-            port = sk.getsockname()[1]
-        cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
-               "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
-        raise SystemExit(subprocess.call(cmd))
+        raise SystemExit(subprocess.call(replica_launch_command(args.gpus, sys.argv[1:])))
     if args.impl == "reference":
         run_reference(args)
     elif args.workload == "decode":

@@ -227,9 +227,9 @@ int gdn_chunk_prefill_gated(const void* q, const void* k, const void* v,
  * after a call that reported GDN_ERR_TIMEOUT set the workspace again before reusing it) and returns GDN_ERR_CUDA if that fails; a pointer that is
  * not 256-byte aligned gives GDN_ERR_UNSUPPORTED.  gdn_set_workspace(NULL, 0) removes it.
  * `packed` is 1 when cu_seqlens will be passed (T = total tokens), else 0.
- * gdn_workspace_bytes returns 0 for sizes the tensor-core path does not support.
+ * gdn_workspace_bytes returns 0 for sizes the tensor-core path does not support (chunk other than 64 included).
  */
-size_t gdn_workspace_bytes(int B, int T, int H, int d_k, int d_v, int packed);
+size_t gdn_workspace_bytes(int B, int T, int H, int d_k, int d_v, int chunk, int packed);
 int gdn_set_workspace(void* device_ptr, size_t bytes);
 
 /*

@@ -13,13 +13,13 @@
 //                          the recurrent layers": S_t = diag(gamma_t) S_{t-1} +
 //                          k_t delta_t^T; state S in R^{H_k x H_v} per value head,
 //                          Section "The model").
-//   gdn_oracle_chunked     the intra-/inter-chunk form of the same section, taken
-//                          in the paper's order: two products form the token-token
-//                          interaction matrices, a forward substitution resolves
-//                          the triangular dependence, products assemble the
-//                          per-chunk correction and output, and a short recurrence
-//                          over chunks carries the state.  form=1 uses the
-//                          section's S^(c+1) = M_c S^(c) + N_c variant.
+//   gdn_oracle_chunked     the intra-/inter-chunk form of the same section, in the order of
+//                          steps the section gives: (1) K K^T and Q K^T of a chunk with
+//                          their decay masks, (2) row-by-row solve of the unit lower
+//                          triangular system, (3) the factors W, U and from them the
+//                          chunk's correction and output, (4) the state carried to the
+//                          next chunk.  form=1 precomputes M_c, N_c per chunk and steps
+//                          with S^(c+1) = M_c S^(c) + N_c, as the section also does.
 //   gdn_oracle_dense       brute force: the whole sequence as one T x T system
 //                          solved by general Gaussian elimination with pivoting
 //                          (it does not know the matrix is triangular).

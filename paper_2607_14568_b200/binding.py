@@ -56,7 +56,7 @@ def lib():
         L.gdn_chunk_prefill_gated.restype = i
         L.gdn_attn_causal_prefill.argtypes = [vp] * 5 + [i] * 5 + [ctypes.c_float, vp]
         L.gdn_attn_causal_prefill.restype = i
-        L.gdn_workspace_bytes.argtypes = [i] * 6
+        L.gdn_workspace_bytes.argtypes = [i] * 7
         L.gdn_workspace_bytes.restype = sz
         L.gdn_set_workspace.argtypes = [vp, sz]
         L.gdn_set_workspace.restype = i
@@ -96,8 +96,8 @@ def gdn_status_string(status: int) -> str:
     return lib().gdn_status_string(int(status)).decode()
 
 
-def gdn_workspace_bytes(B: int, T: int, H: int, d_k: int, d_v: int, packed: bool = False) -> int:
-    return int(lib().gdn_workspace_bytes(B, T, H, d_k, d_v, 1 if packed else 0))
+def gdn_workspace_bytes(B: int, T: int, H: int, d_k: int, d_v: int, packed: bool = False, chunk: int = 64) -> int:
+    return int(lib().gdn_workspace_bytes(B, T, H, d_k, d_v, int(chunk), 1 if packed else 0))
 
 
 _workspace_ref = None

@@ -329,7 +329,8 @@ int gdn_chunk_prefill_gated(const void* q, const void* k, const void* v, const f
     return launch_lean(a, ws.ptr, ws.bytes, reinterpret_cast<cudaStream_t>(stream), opt);
 }
 
-size_t gdn_workspace_bytes(int B, int T, int H, int d_k, int d_v, int packed) {
+size_t gdn_workspace_bytes(int B, int T, int H, int d_k, int d_v, int chunk, int packed) {
+    if (chunk != kChunk) return 0;
     return lean_workspace_bytes(B, T, H, d_k, d_v, packed != 0);
 }
 

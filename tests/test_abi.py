@@ -95,3 +95,15 @@ def test_widened_entry_points_reject_bad_arguments_without_a_gpu(libpath):
     assert snap(p, p, p, p, p, None, p, None, 1, 128, 1, 128, 128, 64, 0, p, None) == 1            # every 0 chunks
     assert snap(p, p, p, p, p, None, p, None, 1, 128, 1, 128, 128, 64, 1, None, None) == 1         # no snapshot buffer
     assert snap(p, p, p, p, p, None, p, None, 1, 128, 1, 128, 128, 64, 1, p, None) == 3            # no workspace set
+
+
+def test_workspace_query_takes_the_chunk_and_rejects_unsupported_tilings(libpath):
+    lib = ctypes.CDLL(libpath)
+    lib.gdn_workspace_bytes.restype = ctypes.c_size_t
+    lib.gdn_workspace_bytes.argtypes = [ctypes.c_int] * 7
+    full = lib.gdn_workspace_bytes(1, 10240, 16, 128, 128, 64, 0)
+    assert full > 160 * 16 * 34048                                 # items of every (chunk, head) plus the split scratch
+    assert lib.gdn_workspace_bytes(1, 10240, 16, 128, 128, 32, 0) == 0      # only 64-token chunks
+    assert lib.gdn_workspace_bytes(1, 10240, 16, 64, 64, 64, 0) == 0        # sizes of the fp32 path need no scratch
+    packed = lib.gdn_workspace_bytes(8, 34000, 16, 128, 128, 64, 1)
+    assert 0 < packed < full * 4

@@ -57,3 +57,16 @@ def test_algorithmic_work_matches_the_stated_formula():
     assert w["tokens"] == 10240
     assert w["flops"] == 10240 * 16 * 180224                      # 6Cd_k + 4Cd_v + 6d_kd_v at d = 128
     assert w["bytes"] == 10240 * 16 * 1032 + 2 * 16 * 128 * 128 * 4
+
+
+def test_bench_starts_its_own_replicas_when_no_launcher_did():
+    """`python bench.py --gpus N` without WORLD_SIZE in the environment must start N ranks itself: the command it
+    builds is the launcher invocation the driver uses (one node, N processes, rendezvous on 127.0.0.1)."""
+    import bench
+    cmd = bench.replica_launch_command(4, ["--gpus", "4", "--steps", "2", "--warmup", "3"], port=29555)
+    assert cmd[1:4] == ["-m", "torch.distributed.run", "--nnodes=1"]
+    assert "--nproc-per-node=4" in cmd and cmd[cmd.index("--master-addr") + 1] == "127.0.0.1"
+    assert cmd[cmd.index("--master-port") + 1] == "29555"
+    assert cmd[-7].endswith("bench.py") and cmd[-6:] == ["--gpus", "4", "--steps", "2", "--warmup", "3"]
+    port = int(bench.replica_launch_command(2, [])[bench.replica_launch_command(2, []).index("--master-port") + 1])
+    assert 1024 < port < 65536
