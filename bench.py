@@ -235,7 +235,8 @@ def run_ours(args):
     if world > 1:
         dist.init_process_group("nccl", device_id=dev)
 
-    cfg = get_config(args.workload)
+    overrides = {k: int(v) for k, v in (kv.split("=") for kv in args.reduce.split(",") if kv)}
+    cfg = get_config(args.workload, **overrides)
     x = make_inputs(cfg)
     work = algorithmic_work(cfg, x.lengths, x.initial_state is not None)
     peaks = measured_peaks()
@@ -395,7 +396,8 @@ def run_ours(args):
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
                 "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True,
                 "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if cfg.dtype == "bf16" else "f32",
-                "data": "synthetic", "config": dict(workload_config(cfg, x), workspace_bytes=int(ws_bytes)),
+                "data": "synthetic", "config": dict(workload_config(cfg, x), workspace_bytes=int(ws_bytes),
+                                                    **({"reduced": args.reduce} if args.reduce else {})),
                 "clocks": clocks, "e2e": e2e,
                 "gpu_launches": int(launches), "roofline": roofline, "cpu_baseline": cpu,
                 "ms_min": float(min(ms)), "ms_median": float(np.median(ms)),
@@ -505,6 +507,8 @@ def main():
                     "attention (T=10240), attention_2k")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-workspace", action="store_true", help="run the fused single-kernel path (no scratch)")
+    ap.add_argument("--reduce", default="", help="profiling only: a reduced copy of the workload, e.g. B=1,T=4096 "
+                    "(the line then names the reduced shape in config; it is not the benchmark configuration)")
     args = ap.parse_args()
     if args.gpus > 1 and "WORLD_SIZE" not in os.environ and args.impl == "ours":
         # not started by a launcher: start one replica process per GPU ourselves (rank 0 prints the line)
