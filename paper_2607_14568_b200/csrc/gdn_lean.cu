@@ -5,7 +5,7 @@
 // sits, once per chunk, on one warpgroup of the few SMs that own a (sequence, head) chain.
 // Here everything that does not depend on the incoming state is taken off those SMs:
 //
-//   gdn_prep_kernel    grid over every (chunk, head), all SMs, three CTAs per SM:
+//   gdn_prep_kernel    every (chunk, head) as an item handed out by a ticket, all SMs, four CTAs per SM:
 //                      step a  cumulative log gate and the gate vectors,
 //                      step b1 G = [K;Q] K^T on the tensor core, decay masks -> A (fp32), P (bf16),
 //                      step b2 T = (I + A)^{-1}, blocked forward substitution in shared memory,
@@ -17,6 +17,11 @@
 //                      TMA brings K, Q, V tiles and the images; U^T = V^T (T diag(b))^T,
 //                      v^T = U^T - S^T W^T, dS^T = (v e^{gC-g})^T K, O^T = e^g S^T Q^T + v^T P^T
 //                      run as tcgen05 MMAs with the state and v_new as TMEM A operands.
+//
+//   gdn_summary_kernel, gdn_combine_kernel   (few chains only) the sequence is cut into segments: per segment
+//                      the map state-in -> state-out is formed from a zero and an identity state, the
+//                      segments' incoming states follow by a short serial walk, and the chain kernel then
+//                      runs all segments at once (see "sequence split" below).
 //
 // (Section "A chunked delta-rule scan for the recurrent layers": state-independent work
 // for all positions at once, then a short recurrence over chunks.)

@@ -30,6 +30,8 @@
 
 #include <cuda.h>
 
+#include <mutex>
+
 #include "gdn_internal.h"
 #include "sm100_ptx.cuh"
 
@@ -760,16 +762,31 @@ EncodeTiledFn encode_fn() {
 }
 
 // [tokens, H, d] bf16, box = 64 tokens x 1 head x 64 features, 128-byte swizzle.
+// A map is a pure function of (address, tokens, H, d): a serving loop calls with the same few buffers again and
+// again, so the last few encodings are kept per host thread and the driver call is skipped on a repeat.
 bool make_map(CUtensorMap* map, const void* ptr, uint64_t tokens, uint64_t H, uint64_t d) {
+    struct Entry { const void* ptr; uint64_t tokens, H, d; CUtensorMap map; bool used; };
+    constexpr int kEntries = 8;
+    static thread_local Entry cache[kEntries] = {};
+    static thread_local int next = 0;
+    for (int i = 0; i < kEntries; ++i)
+        if (cache[i].used && cache[i].ptr == ptr && cache[i].tokens == tokens && cache[i].H == H && cache[i].d == d) {
+            *map = cache[i].map;
+            return true;
+        }
     EncodeTiledFn fn = encode_fn();
     if (!fn) return false;
     const cuuint64_t dims[3] = {d, H, tokens};
     const cuuint64_t strides[2] = {d * 2, H * d * 2};
     const cuuint32_t box[3] = {64, 1, 64};
     const cuuint32_t estr[3] = {1, 1, 1};
-    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    if (fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, estr,
+           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return false;
+    cache[next] = Entry{ptr, tokens, H, d, *map, true};
+    next = (next + 1) % kEntries;
+    return true;
 }
 
 }  // namespace
@@ -800,8 +817,20 @@ int launch_tc(const PrefillArgs& a, cudaStream_t stream) {
         !make_map(&mv, a.v, tokens, a.H, a.d_v))
         return GDN_ERR_CUDA;
     auto kernel = g_debug_dump ? gdn_tc_kernel<true> : gdn_tc_kernel<false>;
-    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES) != cudaSuccess)
-        return GDN_ERR_CUDA;
+    {   // the shared-memory opt-in is a per-device attribute of the kernel: set once per device and variant
+        static std::mutex mu;
+        static bool done[64][2] = {};
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess) return GDN_ERR_CUDA;
+        if (dev < 0 || dev >= 64) return GDN_ERR_UNSUPPORTED;
+        std::lock_guard<std::mutex> lock(mu);
+        const int variant = g_debug_dump ? 1 : 0;
+        if (!done[dev][variant]) {
+            if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES) != cudaSuccess)
+                return GDN_ERR_CUDA;
+            done[dev][variant] = true;
+        }
+    }
     TcParams p{a.log_alpha, a.beta, a.initial_state, static_cast<__nv_bfloat16*>(a.out), a.final_state,
                a.cu_seqlens, g_debug_dump, a.B, a.T, a.H, a.d_v};
     dim3 grid(a.d_v / DVB, a.H, a.B), block(NTHREADS);
