@@ -427,12 +427,20 @@ def run_decode(args):
     for _ in range(max(args.warmup, 3)):
         gdn.gdn_decode_step(q, k, v, la, be, state, out)
     torch.cuda.synchronize()
+    sampler = ClockSampler(int(os.environ.get("LOCAL_RANK", "0")))
+    sampler.start()
+    time.sleep(0.25)
+    l0 = gdn.gdn_launch_count()
+    t0 = time.time()
     for a, b in ev:
         flush.fill_(1)
         a.record()
         gdn.gdn_decode_step(q, k, v, la, be, state, out)
         b.record()
     torch.cuda.synchronize()
+    t1 = time.time()
+    launches = gdn.gdn_launch_count() - l0
+    clocks = sampler.stop(t0, t1)
     ms = float(np.mean([a.elapsed_time(b) for a, b in ev]))
     nbytes = 2 * B * H * dk * dv * 4 + B * H * ((2 * dk + 2 * dv) * 2 + 8)
     peaks = measured_peaks()
@@ -440,7 +448,9 @@ def run_decode(args):
     print(json.dumps({"metric": "gdn_decode_step_tokens_per_s", "value": B / (ms * 1e-3), "unit": "tokens/s",
                       "n_gpus": 1, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms,
                       "higher_is_better": True, "dtype": "f32", "data": "synthetic",
-                      "config": {"workload": "decode", "B": B, "H": H, "d_k": dk, "d_v": dv},
+                      "config": {"workload": "decode", "B": B, "H": H, "d_k": dk, "d_v": dv,
+                                 "l2": "flushed between timed steps (256 MiB write)"},
+                      "clocks": clocks, "gpu_launches": int(launches),
                       "roofline": {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                                    "frac": gbs / peaks["hbm_gbs"], "traffic": None, "peak_source": peaks["source"],
                                    "kernel": "gdn_decode_kernel", "algorithmic_bytes": nbytes}}), flush=True)
@@ -463,12 +473,18 @@ def run_attention(args):
     for _ in range(max(args.warmup, 3)):
         gdn.gdn_attn_causal_prefill(q, k, v, out, cfg.scale)
     torch.cuda.synchronize()
+    sampler = ClockSampler(int(os.environ.get("LOCAL_RANK", "0")))
+    sampler.start()
+    time.sleep(0.25)
+    t0 = time.time()
     for a, b in ev:
         flush.fill_(1)
         a.record()
         gdn.gdn_attn_causal_prefill(q, k, v, out, cfg.scale)
         b.record()
     torch.cuda.synchronize()
+    t1 = time.time()
+    clocks = sampler.stop(t0, t1)
     assert gdn.gdn_query_status() == 0
     ms = float(np.mean([a.elapsed_time(b) for a, b in ev]))
     # algorithmic flops: two products of 2*d flops per (query, visible key) pair and query head
@@ -480,7 +496,7 @@ def run_attention(args):
                       "ms_per_step": ms, "higher_is_better": True, "dtype": "bf16", "data": "synthetic",
                       "config": {"workload": name, "B": cfg.B, "T": cfg.T, "Hq": cfg.Hq, "Hkv": cfg.Hkv, "d": cfg.d,
                                  "l2": "flushed between timed steps (256 MiB write)"},
-                      "gpu_launches": args.steps,
+                      "clocks": clocks, "gpu_launches": args.steps,
                       "roofline": {"bound": "tensor", "achieved": tf, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
                                    "frac": tf / peaks["bf16_tflops"], "traffic": None, "peak_source": peaks["source"],
                                    "kernel": "attn_causal_kernel", "algorithmic_flops": flops}}), flush=True)
