@@ -1436,14 +1436,15 @@ gdn_summary_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
 constexpr int CMB_COLS = 16;                           // value columns per CTA.  Measured on the 10240-token workload: a hop takes
                                                        // about 1.0 us + 0.05 us per column (each thread converts, stores and
                                                        // reloads its own row), so narrow slices on many SMs win
-constexpr int CMB_THREADS = 160;                       // warps 0-3: one state row per thread; warp 4: copies and MMA issue
+constexpr int CMB_THREADS = 224;                       // warps 0-3: one state row per thread; warps 4-6: one MMA issue thread per partial product
 constexpr uint32_t CMB_STAGES = 3;
 constexpr uint32_t CMB_BIMG = CMB_COLS * 256;          // one image of the state slice: [column][row m], two 64-row blocks
 constexpr uint32_t CM_B = CMB_STAGES * CMB_IMG;        // state slice images: leading part | remainder
 constexpr uint32_t CM_BARS = CM_B + 2 * CMB_BIMG;
 constexpr uint32_t CM_MISC = CM_BARS + 16 * 8;
 constexpr uint32_t CMB_SMEM = CM_MISC + 64 + 1024;
-constexpr uint32_t CMB_TCOLS = CMB_COLS < 32 ? 32 : CMB_COLS;
+constexpr uint32_t CMB_TCOLS = 64;                     // three accumulators of CMB_COLS columns (one per partial product)
+static_assert(3 * CMB_COLS <= CMB_TCOLS, "accumulators of the three partial products");
 enum MBar : uint32_t { MB_FULL0 = 0, MB_FREE0 = 3, MB_BREADY = 6, MB_D = 7 };
 constexpr uint32_t ID_CMB = make_idesc(128, CMB_COLS, kFmtBF16, kFmtBF16, kMajorMN, kMajorK);
 
@@ -1456,9 +1457,9 @@ struct CombineParams {
 };
 
 __device__ __forceinline__ void combine_init_bars(const Waiter& w) {
-    for (uint32_t i = 0; i < CMB_STAGES; ++i) { mbar_init(w.bar(MB_FULL0 + i), 1); mbar_init(w.bar(MB_FREE0 + i), 1); }
+    for (uint32_t i = 0; i < CMB_STAGES; ++i) { mbar_init(w.bar(MB_FULL0 + i), 1); mbar_init(w.bar(MB_FREE0 + i), 3); }
     mbar_init(w.bar(MB_BREADY), 128);
-    mbar_init(w.bar(MB_D), 1);
+    mbar_init(w.bar(MB_D), 3);                             // one commit per issue thread
 }
 
 // The hops of one column slice (cta.dvb = slice, cta.z = sequence).  Warps 0-3 own the rows, lane 0 of warp
@@ -1515,22 +1516,28 @@ __device__ __forceinline__ void combine_body(const CombineParams& p, const Cta& 
             tc_fence_after_sync();
 #pragma unroll
             for (int q = 0; q < CMB_COLS / 16; ++q) {
-                uint32_t d[16];
+                uint32_t d[16], e1[16], e2[16];              // hi*hi, lo*hi, hi*lo: one accumulator each
                 tmem_ld16(tmem + lane_base + 16 * q, d);
+                tmem_ld16(tmem + lane_base + CMB_COLS + 16 * q, e1);
+                tmem_ld16(tmem + lane_base + 2 * CMB_COLS + 16 * q, e2);
                 tmem_wait_ld();
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
                     const float4 x = nv[4 * q + e];
-                    s[16 * q + 4 * e + 0] = __uint_as_float(d[4 * e + 0]) + x.x;
-                    s[16 * q + 4 * e + 1] = __uint_as_float(d[4 * e + 1]) + x.y;
-                    s[16 * q + 4 * e + 2] = __uint_as_float(d[4 * e + 2]) + x.z;
-                    s[16 * q + 4 * e + 3] = __uint_as_float(d[4 * e + 3]) + x.w;
+                    const float xs[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+                    for (int u = 0; u < 4; ++u)
+                        s[16 * q + 4 * e + u] = (__uint_as_float(d[4 * e + u]) +
+                                                 (__uint_as_float(e1[4 * e + u]) + __uint_as_float(e2[4 * e + u]))) + xs[u];
                 }
             }
         }
         store_sin(nhops);
-    } else if (warp == issue_warp && lane == 0) {
-        // ---- bulk copies of the M images and MMA issue ----
+    } else if (warp >= issue_warp && warp < issue_warp + 3 && lane == 0) {
+        // ---- MMA issue, one thread per partial product (issuing costs tens of nanoseconds per instruction and the
+        //      three products are independent); the first of them also copies the M images ----
+        const uint32_t prod = (uint32_t)(warp - issue_warp);            // hi*hi, lo*hi, hi*lo
+        const uint32_t aoff = (prod == 1) ? CMB_IMG / 2 : 0u, boff = (prod == 2) ? CMB_BIMG : 0u;
         if (!SCAN) pdl_wait();
         auto load_m = [&](int seg) {
             const uint32_t st = seg % CMB_STAGES, full = w.bar(MB_FULL0 + st);
@@ -1539,29 +1546,26 @@ __device__ __forceinline__ void combine_body(const CombineParams& p, const Cta& 
 #pragma unroll
             for (uint32_t q = 0; q < 4; ++q) bulk_load(base + st * CMB_IMG + q * 16384, src + q * 16384, 16384, full);
         };
-        for (int sg = 0; sg < (int)CMB_STAGES && sg < nhops; ++sg) load_m(sg);
-        const uint64_t dB0 = make_smem_desc(base + CM_B, 16, 1024);
+        if (prod == 0)
+            for (int sg = 0; sg < (int)CMB_STAGES && sg < nhops; ++sg) load_m(sg);
+        const uint64_t dB0 = make_smem_desc(base + CM_B + boff, 16, 1024);
         for (int seg = 0; seg < nhops; ++seg) {
-            const uint32_t st = seg % CMB_STAGES, ma = base + st * CMB_IMG;
+            const uint32_t st = seg % CMB_STAGES, ma = base + st * CMB_IMG + aoff;
             w.wait_hot(MB_FULL0 + st, (seg / CMB_STAGES) & 1);
             w.wait_hot(MB_BREADY, seg & 1);
             tc_fence_after_sync();
 #pragma unroll
-            for (uint32_t prod = 0; prod < 3; ++prod) {          // hi*hi, lo*hi, hi*lo
-                const uint32_t aoff = (prod == 1) ? CMB_IMG / 2 : 0u, boff = (prod == 2) ? CMB_BIMG : 0u;
-#pragma unroll
-                for (uint32_t ks = 0; ks < 8; ++ks)
-                    mma_ss(tmem, make_smem_desc(ma + aoff + (ks >> 2) * 16384 + (ks & 3) * 2048, 8192, 1024),
-                           dB0 + (uint64_t)((boff + (ks >> 2) * (CMB_COLS * 128) + (ks & 3) * 32) >> 4), ID_CMB, (prod | ks) ? 1u : 0u);
-            }
+            for (uint32_t ks = 0; ks < 8; ++ks)
+                mma_ss(tmem + prod * CMB_COLS, make_smem_desc(ma + (ks >> 2) * 16384 + (ks & 3) * 2048, 8192, 1024),
+                       dB0 + (uint64_t)(((ks >> 2) * (CMB_COLS * 128) + (ks & 3) * 32) >> 4), ID_CMB, ks ? 1u : 0u);
             mma_commit(w.bar(MB_D));
             mma_commit(w.bar(MB_FREE0 + st));
-            if (seg + (int)CMB_STAGES < nhops) {
-                w.wait(MB_FREE0 + st, (seg / CMB_STAGES) & 1);   // the tensor core has read this stage
+            if (prod == 0 && seg + (int)CMB_STAGES < nhops) {
+                w.wait(MB_FREE0 + st, (seg / CMB_STAGES) & 1);   // the tensor core has read this stage for all three products
                 load_m(seg + CMB_STAGES);
             }
         }
-        if (*w.abort_flag) {             // let copies in flight land before shared memory is released (bounded)
+        if (prod == 0 && *w.abort_flag) {   // let copies in flight land before shared memory is released (bounded)
             const unsigned long long t0 = globaltimer_ns();
             for (int seg = max(0, nhops - (int)CMB_STAGES); seg < nhops; ++seg)
                 while (!mbar_try_wait(w.bar(MB_FULL0 + seg % CMB_STAGES), (seg / CMB_STAGES) & 1) &&
